@@ -1,0 +1,16 @@
+"""Float64 CPU oracle for SWAA attention.  TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the GPU library never does, and this package never imports the GPU
+library.  See ``swaa_oracle.c`` for the definition it implements and the paper
+passages it follows.
+"""
+from .swaa_oracle import (  # noqa: F401
+    build,
+    count_pairs,
+    decode,
+    layer_is_full,
+    num_threads,
+    prefill,
+    visible,
+)

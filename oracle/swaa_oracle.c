@@ -1,0 +1,217 @@
+/*
+ * swaa_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * Plain, slow, float64 CPU statement of the attention that the SWAA method
+ * computes: causal softmax attention under a per-layer mask policy.  It exists
+ * so that the GPU library can be checked against something written directly
+ * from the paper's definition.  It shares no code with the GPU path and is
+ * only ever called by tests, the smoke check and the benchmark's CPU-baseline
+ * leg.
+ *
+ * What the paper fixes (all in prose; it prints no formula):
+ *   - Sec. 1 / App. A: sliding window attention restricts each token to a
+ *     fixed-size local window of earlier tokens (causal), cost O(N*W).
+ *   - Sec. 3.2.1 "Keep First k Tokens" and the Fig. 1(b) caption: a token
+ *     attends to its local window AND the first k tokens (a union).
+ *   - Sec. 3.1.1 "FA Decode" and the Fig. 1(a) caption: a generated token
+ *     attends to every earlier token of the whole context.
+ *   - Sec. 3.1.2 "Interleaving FA/SWA layers": some layers keep full causal
+ *     attention.
+ *   - Sec. 4.1.2: SWA equals full attention when the context fits the window.
+ *
+ * Readings taken where the paper is silent:
+ *   - the window holds W keys INCLUDING the query's own position:
+ *        visible(i, j) = j <= i  and ( is_full  or  j > i - W  or  j < S )
+ *   - sink positions are relative to the start of each packed sequence;
+ *   - grouped-query attention: query head h reads key/value head h / (Hq/Hkv);
+ *   - the softmax scale is an argument (callers pass 1/sqrt(D));
+ *   - decode: the cache already holds the current token, the query sits at
+ *     position len-1.
+ *
+ * Every row is computed by the textbook two-pass softmax over exactly the
+ * visible keys; keys that are not visible are never read.  No tiling, no
+ * running maximum, no reordering.  Inputs are float32 arrays that hold the
+ * bf16 input values exactly; all arithmetic is double.
+ *
+ * Pins (tests/test_oracle_pins.py): brute-force set enumeration on tiny
+ * inputs, the closed-form visible-pair count, W >= L == full causal (Sec.
+ * 4.1.2) == a library float64 softmax-attention, W=1/S=0 returns V, Q=0
+ * returns the mean of the visible V rows, rows of probabilities sum to 1,
+ * decode == last prefill row.  No value printed by the paper exists to
+ * compare against (it prints none for this path).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* Sec. 3.2.1 (window AND first k), Sec. 1 (causal local window), Sec. 3.1.1/3.1.2 (full). */
+int swaa_oracle_visible(int64_t i, int64_t j, int64_t W, int64_t S, int is_full) {
+    if (j < 0 || j > i) return 0;   /* causal */
+    if (is_full) return 1;          /* FA layer or FA decode */
+    if (j > i - W) return 1;        /* inside the window of W keys ending at i */
+    if (j < S) return 1;            /* one of the first S (sink) tokens */
+    return 0;
+}
+
+/* Number of visible (i, j) pairs of one sequence of length L, by direct enumeration. */
+int64_t swaa_oracle_count_pairs(int64_t L, int64_t W, int64_t S, int is_full) {
+    int64_t n = 0;
+    for (int64_t i = 0; i < L; ++i)
+        for (int64_t j = 0; j <= i; ++j)
+            n += swaa_oracle_visible(i, j, W, S, is_full);
+    return n;
+}
+
+/*
+ * One output row.  q: D values of the query at position i of its sequence.
+ * k, v: position 0 of the same sequence and key/value head; consecutive
+ * positions are kv_stride floats apart.  Writes out[D]; *lse = log of the sum
+ * of exp(score) over visible keys; *psum = sum of the normalised probabilities
+ * (should be 1); *nvis = how many keys were visible.  `scores` is scratch of at
+ * least i+1 doubles.
+ */
+static void oracle_row(const float* q, const float* k, const float* v, int64_t i, int64_t kv_stride, int D,
+                       int64_t W, int64_t S, int is_full, double scale, double* out, double* lse, double* psum,
+                       int64_t* nvis, double* scores) {
+    double m = -INFINITY;
+    int64_t cnt = 0;
+    for (int64_t j = 0; j <= i; ++j) {
+        if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+        const float* kj = k + j * kv_stride;
+        double s = 0.0;
+        for (int d = 0; d < D; ++d) s += (double)q[d] * (double)kj[d];
+        s *= scale;
+        scores[j] = s;
+        if (s > m) m = s;
+        ++cnt;
+    }
+    for (int d = 0; d < D; ++d) out[d] = 0.0;
+    double denom = 0.0;
+    for (int64_t j = 0; j <= i; ++j) {
+        if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+        denom += exp(scores[j] - m);
+    }
+    double ps = 0.0;
+    for (int64_t j = 0; j <= i; ++j) {
+        if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+        double p = exp(scores[j] - m) / denom;
+        ps += p;
+        const float* vj = v + j * kv_stride;
+        for (int d = 0; d < D; ++d) out[d] += p * (double)vj[d];
+    }
+    if (lse) *lse = m + log(denom);
+    if (psum) *psum = ps;
+    if (nvis) *nvis = cnt;
+}
+
+/*
+ * Packed variable-length prefill (self attention, one cu_seqlens for q and k).
+ *   q   [T, Hq, D], k, v [T, Hkv, D]  float32 (bf16 values), token-major.
+ *   cu_seqlens [B+1], cu[0] = 0, cu[B] = T.
+ * Computes n_rows rows chosen by (row_t[r], row_h[r]) = (packed token index,
+ * query head); with row_t == NULL every (t, h) is computed in t-major order and
+ * n_rows must be T*Hq.  out is [n_rows, D] double; lse, psum, nvis are
+ * [n_rows] (each may be NULL).  Returns 0, or -1 on inconsistent arguments.
+ */
+int swaa_oracle_prefill(const float* q, const float* k, const float* v, const int32_t* cu_seqlens, int B, int Hq,
+                        int Hkv, int D, int64_t W, int64_t S, int is_full, double scale, int64_t n_rows,
+                        const int64_t* row_t, const int32_t* row_h, double* out, double* lse, double* psum,
+                        int64_t* nvis) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
+    if (!is_full && W < 1) return -1;
+    if (S < 0) return -1;
+    const int G = Hq / Hkv;
+    const int64_t T = B > 0 ? cu_seqlens[B] : 0;
+    int64_t max_len = 0;
+    for (int b = 0; b < B; ++b) {
+        int64_t len = (int64_t)cu_seqlens[b + 1] - cu_seqlens[b];
+        if (len < 0) return -1;
+        if (len > max_len) max_len = len;
+    }
+    if (row_t == NULL && n_rows != T * Hq) return -1;
+    int bad = 0;
+#pragma omp parallel
+    {
+        double* scores = (double*)malloc(sizeof(double) * (size_t)(max_len > 0 ? max_len : 1));
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            int64_t t = row_t ? row_t[r] : r / Hq;
+            int h = row_t ? row_h[r] : (int)(r % Hq);
+            if (t < 0 || t >= T || h < 0 || h >= Hq) { bad = 1; continue; }
+            int b = 0;
+            while (!(cu_seqlens[b] <= t && t < cu_seqlens[b + 1])) ++b; /* sequence that owns token t */
+            int64_t start = cu_seqlens[b];
+            int64_t i = t - start; /* position inside its own sequence */
+            int hk = h / G;
+            oracle_row(q + (t * Hq + h) * (int64_t)D, k + (start * Hkv + hk) * (int64_t)D,
+                       v + (start * Hkv + hk) * (int64_t)D, i, (int64_t)Hkv * D, D, W, S, is_full, scale,
+                       out + r * D, lse ? lse + r : NULL, psum ? psum + r : NULL, nvis ? nvis + r : NULL, scores);
+        }
+        free(scores);
+    }
+    return bad ? -1 : 0;
+}
+
+/*
+ * Decode: one query token per sequence against a dense cache.
+ *   q [B, Hq, D]; kcache, vcache [B, Lmax, Hkv, D]; seqlens [B] counts the valid
+ *   cache entries INCLUDING the current token, so the query's position is
+ *   seqlens[b]-1 (Sec. 3.1.1: with is_full it sees the whole context).
+ * out [B, Hq, D] double; lse, psum, nvis [B, Hq] (nullable).
+ */
+int swaa_oracle_decode(const float* q, const float* kcache, const float* vcache, const int32_t* seqlens, int B,
+                       int64_t Lmax, int Hq, int Hkv, int D, int64_t W, int64_t S, int is_full, double scale,
+                       double* out, double* lse, double* psum, int64_t* nvis) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
+    if (!is_full && W < 1) return -1;
+    if (S < 0) return -1;
+    const int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b)
+        if (seqlens[b] < 1 || seqlens[b] > Lmax) return -1;
+#pragma omp parallel
+    {
+        double* scores = (double*)malloc(sizeof(double) * (size_t)(Lmax > 0 ? Lmax : 1));
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t r = 0; r < (int64_t)B * Hq; ++r) {
+            int b = (int)(r / Hq), h = (int)(r % Hq), hk = h / G;
+            int64_t i = (int64_t)seqlens[b] - 1;
+            oracle_row(q + r * D, kcache + ((int64_t)b * Lmax * Hkv + hk) * D,
+                       vcache + ((int64_t)b * Lmax * Hkv + hk) * D, i, (int64_t)Hkv * D, D, W, S, is_full, scale,
+                       out + r * D, lse ? lse + r : NULL, psum ? psum + r : NULL, nvis ? nvis + r : NULL, scores);
+        }
+        free(scores);
+    }
+    return 0;
+}
+
+/*
+ * Layer schedule (Sec. 3.1.2 fixed-interval FA layers; Sec. 3.1.1 FA decode;
+ * Table 1 columns "FA layers" and "FA decode").  Layers fa_start, fa_start +
+ * fa_step, ... keep full attention (fa_step == 0: none).  phase 0 = prefill,
+ * 1 = decode.  With fa_decode every layer is full in the decode phase.
+ */
+int swaa_oracle_layer_is_full(int layer, int fa_start, int fa_step, int fa_decode, int phase) {
+    int in_list = 0;
+    if (fa_step > 0)
+        for (int l = fa_start; l <= layer; l += fa_step)
+            if (l == layer) in_list = 1;
+    if (in_list) return 1;
+    if (phase == 1 && fa_decode) return 1;
+    return 0;
+}
+
+int swaa_oracle_num_threads(void) {
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp single
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}

@@ -1,0 +1,139 @@
+"""ctypes front end of the plain-C float64 oracle.  TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+
+Marshals numpy arrays into ``swaa_oracle.c`` and nothing else: every number the
+oracle returns is computed by the C file's plain loops.  Inputs are float32 (or
+anything convertible) arrays holding the bf16 input values exactly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "swaa_oracle.c")
+_SO = os.path.join(_HERE, "libswaa_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP over rows) if it is missing or stale."""
+    with _lock:
+        stale = (not os.path.exists(_SO)) or os.path.getmtime(_SO) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _SO + f".tmp{os.getpid()}"
+            subprocess.check_call(
+                ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-Wall", "-o", tmp, _SRC, "-lm"]
+            )
+            os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, i32, dbl, vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p
+        lib.swaa_oracle_visible.argtypes = [i64, i64, i64, i64, ctypes.c_int]
+        lib.swaa_oracle_visible.restype = ctypes.c_int
+        lib.swaa_oracle_count_pairs.argtypes = [i64, i64, i64, ctypes.c_int]
+        lib.swaa_oracle_count_pairs.restype = i64
+        lib.swaa_oracle_prefill.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl, i64,
+                                            vp, vp, vp, vp, vp, vp]
+        lib.swaa_oracle_prefill.restype = ctypes.c_int
+        lib.swaa_oracle_decode.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
+                                           vp, vp, vp, vp]
+        lib.swaa_oracle_decode.restype = ctypes.c_int
+        lib.swaa_oracle_layer_is_full.argtypes = [ctypes.c_int] * 5
+        lib.swaa_oracle_layer_is_full.restype = ctypes.c_int
+        lib.swaa_oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def visible(i: int, j: int, W: int, S: int, is_full: bool) -> bool:
+    return bool(_load().swaa_oracle_visible(i, j, W, S, int(bool(is_full))))
+
+
+def count_pairs(L: int, W: int, S: int, is_full: bool) -> int:
+    return int(_load().swaa_oracle_count_pairs(L, W, S, int(bool(is_full))))
+
+
+def num_threads() -> int:
+    return int(_load().swaa_oracle_num_threads())
+
+
+def layer_is_full(layer: int, fa_start: int, fa_step: int, fa_decode: bool, phase: int) -> bool:
+    return bool(_load().swaa_oracle_layer_is_full(layer, fa_start, fa_step, int(bool(fa_decode)), phase))
+
+
+def prefill(q, k, v, cu_seqlens, window: int, n_sink: int, is_full: bool, scale: float | None = None, rows=None):
+    """Packed varlen prefill.  q [T,Hq,D]; k, v [T,Hkv,D]; cu_seqlens [B+1].
+
+    rows: optional (row_t, row_h) integer arrays selecting (packed token, q-head)
+    rows; default all rows in token-major order.  Returns a dict with
+    out [n_rows, D] (or [T,Hq,D] for all rows), lse, psum, nvis.
+    """
+    q, k, v = _f32(q), _f32(k), _f32(v)
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == (T, Hkv, D) and v.shape == (T, Hkv, D)
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    B = cu.shape[0] - 1
+    assert cu[0] == 0 and cu[-1] == T
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    if rows is None:
+        n_rows, rt, rh = T * Hq, None, None
+    else:
+        rt = np.ascontiguousarray(np.asarray(rows[0], dtype=np.int64))
+        rh = np.ascontiguousarray(np.asarray(rows[1], dtype=np.int32))
+        n_rows = rt.shape[0]
+        assert rh.shape[0] == n_rows
+    out = np.empty((n_rows, D), dtype=np.float64)
+    lse = np.empty(n_rows, dtype=np.float64)
+    psum = np.empty(n_rows, dtype=np.float64)
+    nvis = np.empty(n_rows, dtype=np.int64)
+    rc = _load().swaa_oracle_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(cu), B, Hq, Hkv, D, int(window), int(n_sink),
+                                     int(bool(is_full)), float(scale), n_rows, _ptr(rt), _ptr(rh), _ptr(out),
+                                     _ptr(lse), _ptr(psum), _ptr(nvis))
+    if rc != 0:
+        raise ValueError("swaa_oracle_prefill: inconsistent arguments")
+    if rows is None:
+        return {"out": out.reshape(T, Hq, D), "lse": lse.reshape(T, Hq), "psum": psum.reshape(T, Hq),
+                "nvis": nvis.reshape(T, Hq)}
+    return {"out": out, "lse": lse, "psum": psum, "nvis": nvis}
+
+
+def decode(q, kcache, vcache, seqlens, window: int, n_sink: int, is_full: bool, scale: float | None = None):
+    """Decode.  q [B,Hq,D]; caches [B,Lmax,Hkv,D]; seqlens [B] (valid entries incl. the current token)."""
+    q, kcache, vcache = _f32(q), _f32(kcache), _f32(vcache)
+    B, Hq, D = q.shape
+    _, Lmax, Hkv, _ = kcache.shape
+    assert kcache.shape == (B, Lmax, Hkv, D) and vcache.shape == kcache.shape
+    sl = np.ascontiguousarray(np.asarray(seqlens, dtype=np.int32))
+    assert sl.shape == (B,)
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    out = np.empty((B, Hq, D), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    psum = np.empty((B, Hq), dtype=np.float64)
+    nvis = np.empty((B, Hq), dtype=np.int64)
+    rc = _load().swaa_oracle_decode(_ptr(q), _ptr(kcache), _ptr(vcache), _ptr(sl), B, Lmax, Hq, Hkv, D,
+                                    int(window), int(n_sink), int(bool(is_full)), float(scale), _ptr(out),
+                                    _ptr(lse), _ptr(psum), _ptr(nvis))
+    if rc != 0:
+        raise ValueError("swaa_oracle_decode: inconsistent arguments")
+    return {"out": out, "lse": lse, "psum": psum, "nvis": nvis}
