@@ -1,0 +1,153 @@
+/*
+ * swaa.h -- C ABI of the SWAA attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes causal softmax attention under the per-layer mask policy
+ * of SWAA ("Sliding Window Attention Adaptation"):
+ *
+ *     visible(i, j) = j <= i  and  ( is_full  or  j > i - window  or  j < n_sink )
+ *
+ * with i, j the positions of query and key inside their own sequence.
+ *   - window: sliding window attention, each token sees a fixed-size local
+ *     window (Sec. 1, App. A); the window counts `window` keys including the
+ *     query's own position.
+ *   - n_sink: "Keep First k Tokens", every token additionally sees the first k
+ *     tokens of its sequence (Sec. 3.2.1, Fig. 1b).
+ *   - is_full: full causal attention, used by FA layers of an interleaved stack
+ *     (Sec. 3.1.2) and by the decode phase under "FA Decode" (Sec. 3.1.1, Fig. 1a).
+ * Grouped-query attention: query head h reads key/value head h / (Hq / Hkv).
+ * Arithmetic: bf16 inputs, fp32 accumulation, bf16 outputs.
+ *
+ * Conventions for every call
+ *   - Pointers named "device" are CUDA device pointers on the current device;
+ *     the caller owns every buffer.  Tensors are dense and contiguous in the
+ *     stated layout, bf16 unless stated, and 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work
+ *     is enqueued asynchronously; no call synchronises except
+ *     swaa_last_device_status.
+ *   - The return value is a swaa_status.  Argument errors are detected on the
+ *     host before anything is launched.  Errors only the device can see (bad
+ *     cu_seqlens / seqlens contents, a bounded wait that ran out) are recorded in
+ *     a per-device status word that swaa_last_device_status reads; a kernel that
+ *     records one skips the stores of the affected rows and returns normally.
+ *   - The library allocates no device memory.  There is no CPU fallback.
+ */
+#ifndef SWAA_H_
+#define SWAA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SWAA_OK = 0,
+    SWAA_ERR_INVALID_ARG = -1, /* null / misaligned pointer, negative size, window < 1 on an SWA call, ... */
+    SWAA_ERR_UNSUPPORTED = -2, /* D not in {64, 128}, Hq % Hkv != 0, device is not sm_100 */
+    SWAA_ERR_CUDA = -3,        /* a CUDA runtime / driver call failed */
+    SWAA_ERR_WORKSPACE = -4,   /* workspace too small or misaligned */
+    SWAA_ERR_BAD_SEQLENS = -5, /* device saw inconsistent cu_seqlens / seqlens */
+    SWAA_ERR_TIMEOUT = -6      /* a bounded device-side wait ran out */
+} swaa_status;
+
+/*
+ * Prefill: packed variable-length causal self attention (Sec. 1, 3.1.2, 3.2.1; App. A: cost O(N*W)).
+ *
+ *   q, out      device, [T, Hq, D]  bf16 (token-major: token, head, channel)
+ *   k, v        device, [T, Hkv, D] bf16
+ *   cu_seqlens  device, int32 [B+1]; cu[0] = 0, cu[B] = T, non-decreasing.  Sequence b owns packed
+ *               tokens cu[b] .. cu[b+1]-1; positions (and the n_sink first tokens) are per sequence.
+ *   B, T        number of sequences, total packed tokens.  T == 0 or B == 0 is a no-op (SWAA_OK).
+ *   max_seqlen  upper bound on any sequence length (sizes the launch); a longer sequence is reported
+ *               as SWAA_ERR_BAD_SEQLENS through the status word and its rows are not written.
+ *   Hq, Hkv, D  head counts and head size; Hq % Hkv == 0; D in {64, 128}.
+ *   window      >= 1 unless is_full; n_sink >= 0; is_full != 0 selects full causal attention
+ *               (window and n_sink are then ignored).
+ *   scale       softmax scale; <= 0 selects 1/sqrt(D).
+ *   lse         device, float32 [Hq, T], natural-log sum of exp(scale * q.k) over the visible keys of
+ *               each row; may be NULL.
+ * Only the key tiles that hold a visible key are visited: the sink tiles and the diagonal band.
+ */
+int swaa_prefill(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens, int B, int T,
+                 int max_seqlen, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
+                 float* lse, void* stream);
+
+/*
+ * Decode: one query token per sequence against a dense KV cache (Sec. 3.1.1 "FA Decode": with is_full
+ * the generated token sees the whole context; App. A: the full-context cache is retained).
+ *
+ *   q, out          device, [B, Hq, D] bf16
+ *   kcache, vcache  device, [B, Lmax, Hkv, D] bf16
+ *   seqlens         device, int32 [B]; number of valid cache entries of each sequence INCLUDING the
+ *                   current token, 1 <= seqlens[b] <= Lmax; the query sits at position seqlens[b]-1.
+ *                   With is_full == 0 it reads the last `window` entries plus the first n_sink.
+ *                   A value outside [1, Lmax] is reported as SWAA_ERR_BAD_SEQLENS through the status
+ *                   word; that sequence's output rows are zero-filled.
+ *   workspace       device scratch of at least swaa_decode_workspace_size(...) bytes for the same
+ *                   shape arguments, 256-byte aligned; contents need not be initialised and are
+ *                   overwritten.  Two calls that overlap on the GPU must not share a workspace.
+ * The visible cache entries are split over thread blocks (split-K); partial results are merged by a
+ * log-sum-exp combine inside the same launch.
+ */
+size_t swaa_decode_workspace_size(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full);
+
+int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens, int B,
+                int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale, void* workspace,
+                size_t workspace_bytes, void* stream);
+
+/*
+ * Layer schedule (host only).  Sec. 3.1.2: a fixed-interval subset of layers keeps full attention
+ * (Table 1 "FA layers": [1,3,5,...], [0,2,4,...], [1,5,9,...], [1,9,17,...], [3,7,11,...]); Sec. 3.1.1:
+ * with FA decode every layer is full while decoding.  Layers are 0-based.
+ *   is_full(layer, phase) = (layer in {fa_start, fa_start+fa_step, ...}) or (phase == decode and fa_decode)
+ */
+typedef struct {
+    int n_layers;
+    int window;    /* SWA window of the non-FA layers */
+    int n_sink;    /* keep-first k */
+    int fa_start;  /* first FA layer */
+    int fa_step;   /* distance between FA layers; 0 = no FA layers */
+    int fa_decode; /* non-zero: full attention in the decode phase on every layer */
+} swaa_policy;
+
+#define SWAA_PHASE_PREFILL 0
+#define SWAA_PHASE_DECODE 1
+
+/* Returns 1 / 0, or SWAA_ERR_INVALID_ARG (null policy, layer outside [0, n_layers), bad phase, negative fields). */
+int swaa_schedule_is_full(const swaa_policy* policy, int layer, int phase);
+/* Fills is_full_out[0 .. n_layers) (host memory) with 0/1.  Returns SWAA_OK or SWAA_ERR_INVALID_ARG. */
+int swaa_schedule_fill(const swaa_policy* policy, int phase, uint8_t* is_full_out);
+
+/*
+ * Key-tile enumeration of the prefill kernel, exposed for host-side verification (App. A: only
+ * O(N*W) work).  For the query tile of rows [m*BM, min(L, (m+1)*BM)) of a sequence of length L, the
+ * kernel visits key tiles (of BN keys) 0 .. *n_sink_tiles-1 and *n_lo .. *n_hi.  Returns SWAA_OK or
+ * SWAA_ERR_INVALID_ARG.  swaa_prefill_tile_needs_mask returns 1 when some (row, key) pair of the
+ * tile is not visible (the kernel then applies the element predicate), 0 when every pair is visible.
+ */
+int swaa_prefill_tile_range(int L, int m, int BM, int BN, int window, int n_sink, int is_full, int* n_sink_tiles,
+                            int* n_lo, int* n_hi);
+int swaa_prefill_tile_needs_mask(int L, int m, int n, int BM, int BN, int window, int n_sink, int is_full);
+/* Tile sizes the prefill kernel uses (rows per query tile, keys per key tile). */
+int swaa_prefill_block_m(void);
+int swaa_prefill_block_n(void);
+
+/* Number of key splits swaa_decode uses for these arguments on the current device (>= 1). */
+int swaa_decode_num_splits(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full);
+
+/* Static string for a swaa_status value. */
+const char* swaa_status_str(int status);
+/*
+ * Waits for `stream` to drain, then returns and clears the current device's status word: SWAA_OK, or
+ * the first device-detected error since the last call (SWAA_ERR_BAD_SEQLENS, SWAA_ERR_TIMEOUT), or
+ * SWAA_ERR_CUDA if the stream itself reports an error.
+ */
+int swaa_last_device_status(void* stream);
+/* Kernels launched by this library in this process so far (all devices, all streams). */
+uint64_t swaa_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWAA_H_ */

@@ -1,0 +1,25 @@
+"""SWAA attention hot path for NVIDIA B200 (sm_100a).
+
+``swaa_prefill`` / ``swaa_decode`` and the host-side layer schedule, as a C-ABI
+shared library (``csrc/``, ``include/swaa.h``) plus this thin ctypes binding.
+The library is loaded on first use; there is no CPU fallback: a missing or
+unloadable library raises.
+"""
+from .binding import (  # noqa: F401
+    SwaaError,
+    SwaaPolicy,
+    decode_num_splits,
+    decode_workspace_size,
+    kernel_launch_count,
+    prefill_block_shape,
+    prefill_tile_needs_mask,
+    prefill_tile_range,
+    lib_path,
+    load_library,
+    schedule_fill,
+    schedule_is_full,
+    status_str,
+    swaa_decode,
+    swaa_prefill,
+    last_device_status,
+)

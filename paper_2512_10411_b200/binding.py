@@ -1,0 +1,205 @@
+"""ctypes binding of libswaa.so: argument marshalling only.
+
+Every function has the name of the C entry point it forwards to (include/swaa.h).  Tensors are
+torch tensors used purely as device-memory handles: the binding checks dtype, device and contiguity,
+reads sizes from the shapes, passes raw pointers, and raises ``SwaaError`` on a non-zero status.
+There is no fallback path: if the shared library is missing or cannot be loaded, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from .build import LIB_PATH
+
+SWAA_OK = 0
+SWAA_PHASE_PREFILL = 0
+SWAA_PHASE_DECODE = 1
+
+_lib = None
+
+
+class SwaaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_str(status)} ({status})")
+
+
+class _Policy(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("n_layers", "window", "n_sink", "fa_start", "fa_step", "fa_decode")]
+
+
+@dataclass
+class SwaaPolicy:
+    """Mirror of the C struct swaa_policy (one SWAA configuration: window, FA layers, keep first, FA decode)."""
+    n_layers: int
+    window: int
+    n_sink: int = 0
+    fa_start: int = 0
+    fa_step: int = 0
+    fa_decode: bool = False
+
+    def _c(self) -> _Policy:
+        return _Policy(self.n_layers, self.window, self.n_sink, self.fa_start, self.fa_step, int(bool(self.fa_decode)))
+
+
+def lib_path() -> str:
+    return LIB_PATH
+
+
+def load_library():
+    """Loads libswaa.so (built in-tree by ``build.build_library``); raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2512_10411_b200.build` "
+                           "(there is no fallback implementation)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    lib.swaa_prefill.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
+    lib.swaa_prefill.restype = ci
+    lib.swaa_decode_workspace_size.argtypes = [ci] * 8
+    lib.swaa_decode_workspace_size.restype = ctypes.c_size_t
+    lib.swaa_decode_num_splits.argtypes = [ci] * 8
+    lib.swaa_decode_num_splits.restype = ci
+    lib.swaa_decode.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
+    lib.swaa_decode.restype = ci
+    lib.swaa_schedule_is_full.argtypes = [ctypes.POINTER(_Policy), ci, ci]
+    lib.swaa_schedule_is_full.restype = ci
+    lib.swaa_schedule_fill.argtypes = [ctypes.POINTER(_Policy), ci, ctypes.POINTER(ctypes.c_uint8)]
+    lib.swaa_schedule_fill.restype = ci
+    lib.swaa_prefill_tile_range.argtypes = [ci] * 7 + [ctypes.POINTER(ci)] * 3
+    lib.swaa_prefill_tile_range.restype = ci
+    lib.swaa_prefill_tile_needs_mask.argtypes = [ci] * 8
+    lib.swaa_prefill_tile_needs_mask.restype = ci
+    lib.swaa_prefill_block_m.restype = ci
+    lib.swaa_prefill_block_n.restype = ci
+    lib.swaa_status_str.argtypes = [ci]
+    lib.swaa_status_str.restype = ctypes.c_char_p
+    lib.swaa_last_device_status.argtypes = [vp]
+    lib.swaa_last_device_status.restype = ci
+    lib.swaa_kernel_launch_count.restype = ctypes.c_uint64
+    _lib = lib
+    return lib
+
+
+def status_str(status: int) -> str:
+    return load_library().swaa_status_str(int(status)).decode()
+
+
+def _dev_ptr(t: torch.Tensor | None, dtype, name: str):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def swaa_prefill(q, k, v, out, cu_seqlens, max_seqlen: int, window: int, n_sink: int, is_full: bool,
+                 scale: float = 0.0, lse=None, stream=None) -> None:
+    """Forwards to C swaa_prefill.  q, out [T,Hq,D]; k, v [T,Hkv,D] bf16; cu_seqlens int32 [B+1]; lse f32 [Hq,T]."""
+    lib = load_library()
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    if tuple(k.shape) != (T, Hkv, D) or tuple(v.shape) != (T, Hkv, D) or tuple(out.shape) != (T, Hq, D):
+        raise ValueError("swaa_prefill: inconsistent tensor shapes")
+    B = cu_seqlens.numel() - 1
+    if lse is not None and tuple(lse.shape) != (Hq, T):
+        raise ValueError("swaa_prefill: lse must be [Hq, T]")
+    bf = torch.bfloat16
+    rc = lib.swaa_prefill(_dev_ptr(q, bf, "q"), _dev_ptr(k, bf, "k"), _dev_ptr(v, bf, "v"), _dev_ptr(out, bf, "out"),
+                          _dev_ptr(cu_seqlens, torch.int32, "cu_seqlens"), B, T, int(max_seqlen), Hq, Hkv, D,
+                          int(window), int(n_sink), int(bool(is_full)), float(scale),
+                          _dev_ptr(lse, torch.float32, "lse"), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_prefill")
+
+
+def decode_workspace_size(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) -> int:
+    """Forwards to C swaa_decode_workspace_size (bytes)."""
+    return int(load_library().swaa_decode_workspace_size(B, Hq, Hkv, D, Lmax, int(window), int(n_sink),
+                                                         int(bool(is_full))))
+
+
+def decode_num_splits(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) -> int:
+    return int(load_library().swaa_decode_num_splits(B, Hq, Hkv, D, Lmax, int(window), int(n_sink),
+                                                     int(bool(is_full))))
+
+
+def swaa_decode(q, kcache, vcache, out, seqlens, window: int, n_sink: int, is_full: bool, workspace,
+                scale: float = 0.0, stream=None) -> None:
+    """Forwards to C swaa_decode.  q, out [B,Hq,D]; caches [B,Lmax,Hkv,D] bf16; seqlens int32 [B];
+    workspace: uint8 CUDA tensor of at least decode_workspace_size(...) bytes."""
+    lib = load_library()
+    B, Hq, D = q.shape
+    _, Lmax, Hkv, _ = kcache.shape
+    if tuple(kcache.shape) != (B, Lmax, Hkv, D) or tuple(vcache.shape) != (B, Lmax, Hkv, D) \
+            or tuple(out.shape) != (B, Hq, D) or seqlens.numel() != B:
+        raise ValueError("swaa_decode: inconsistent tensor shapes")
+    bf = torch.bfloat16
+    rc = lib.swaa_decode(_dev_ptr(q, bf, "q"), _dev_ptr(kcache, bf, "kcache"), _dev_ptr(vcache, bf, "vcache"),
+                         _dev_ptr(out, bf, "out"), _dev_ptr(seqlens, torch.int32, "seqlens"), B, Lmax, Hq, Hkv, D,
+                         int(window), int(n_sink), int(bool(is_full)), float(scale),
+                         _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_decode")
+
+
+def schedule_is_full(policy: SwaaPolicy, layer: int, phase: int) -> bool:
+    c = policy._c()
+    rc = load_library().swaa_schedule_is_full(ctypes.byref(c), int(layer), int(phase))
+    if rc < 0:
+        raise SwaaError(rc, "swaa_schedule_is_full")
+    return bool(rc)
+
+
+def schedule_fill(policy: SwaaPolicy, phase: int) -> list:
+    c = policy._c()
+    buf = (ctypes.c_uint8 * max(policy.n_layers, 1))()
+    rc = load_library().swaa_schedule_fill(ctypes.byref(c), int(phase), buf)
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_schedule_fill")
+    return [bool(buf[i]) for i in range(policy.n_layers)]
+
+
+def prefill_tile_range(L, m, BM, BN, window, n_sink, is_full):
+    a, b, c = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    rc = load_library().swaa_prefill_tile_range(L, m, BM, BN, int(window), int(n_sink), int(bool(is_full)),
+                                                ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_prefill_tile_range")
+    return a.value, b.value, c.value
+
+
+def prefill_tile_needs_mask(L, m, n, BM, BN, window, n_sink, is_full) -> bool:
+    rc = load_library().swaa_prefill_tile_needs_mask(L, m, n, BM, BN, int(window), int(n_sink), int(bool(is_full)))
+    if rc < 0:
+        raise SwaaError(rc, "swaa_prefill_tile_needs_mask")
+    return bool(rc)
+
+
+def prefill_block_shape():
+    lib = load_library()
+    return lib.swaa_prefill_block_m(), lib.swaa_prefill_block_n()
+
+
+def last_device_status(stream=None) -> int:
+    return int(load_library().swaa_last_device_status(_stream_ptr(stream)))
+
+
+def kernel_launch_count() -> int:
+    return int(load_library().swaa_kernel_launch_count())

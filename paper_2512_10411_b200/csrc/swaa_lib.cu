@@ -1,0 +1,252 @@
+// libswaa: C-ABI entry points (see include/swaa.h).  Host-side validation, planning and launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "swaa.h"
+#include "swaa_internal.cuh"
+#include "swaa_decode.cuh"
+#include "swaa_prefill.cuh"
+
+namespace swaa {
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceInfo {
+    bool known = false;
+    int sm_count = 0;
+    int cc_major = 0;
+};
+
+// Properties of the current device, queried once per device.
+static int current_device_info(DeviceInfo* out) {
+    static std::mutex mu;
+    static DeviceInfo table[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SWAA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!table[dev].known) {
+        int sms = 0, major = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SWAA_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return SWAA_ERR_CUDA;
+        table[dev].sm_count = sms;
+        table[dev].cc_major = major;
+        table[dev].known = true;
+    }
+    *out = table[dev];
+    return SWAA_OK;
+}
+
+// ------------------------------------------------------------------------------------------ decode
+struct DecodePlan {
+    int NH;        // 8-head blocks per chunk (1 or 2)
+    int HG;        // chunks per kv head
+    int nsplit;
+    size_t off_ml, off_o, bytes;
+};
+
+// Chooses the number of key splits so that the grid fills the machine in whole waves while every
+// block still streams a few hundred keys.  Depends only on the shape arguments and the SM count.
+static DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full,
+                              int sm_count) {
+    DecodePlan pl;
+    const int G = Hq / Hkv;
+    pl.NH = G > 8 ? 2 : 1;
+    const int HC = 8 * pl.NH;
+    pl.HG = (G + HC - 1) / HC;
+    long long n_vis_max = Lmax;
+    if (!is_full) {
+        long long ws = (long long)window + (long long)n_sink;
+        if (ws < n_vis_max) n_vis_max = ws;
+    }
+    const long long nblk = (n_vis_max + kDecodeBlockKeys - 1) / kDecodeBlockKeys;
+    const long long base = (long long)B * Hkv * pl.HG;
+    const long long capacity = (long long)(sm_count > 0 ? sm_count : 148) * 2;  // resident blocks
+    const long long min_blocks_per_split = 4LL * kDecodeWarps;                  // >= 256 keys per block
+    long long max_ns = nblk / min_blocks_per_split;
+    if (max_ns < 1) max_ns = 1;
+    if (max_ns > 64) max_ns = 64;
+    int best = 1;
+    double best_score = -1.0;
+    for (long long ns = 1; ns <= max_ns; ++ns) {
+        const double waves = (double)(base * ns) / (double)capacity;
+        const double eff = waves / ceil(waves);
+        // prefer full waves; among equals prefer more (smaller) blocks up to about four waves
+        const double score = eff + 0.02 * (waves < 4.0 ? waves : 4.0);
+        if (score > best_score + 1e-9) {
+            best_score = score;
+            best = (int)ns;
+        }
+    }
+    pl.nsplit = best;
+    const size_t counters = ((size_t)base * sizeof(int) + 255) / 256 * 256;
+    const size_t ml = (((size_t)B * Hq * pl.nsplit * 2 * sizeof(float)) + 255) / 256 * 256;
+    const size_t o = (size_t)B * Hq * pl.nsplit * D * sizeof(float);
+    pl.off_ml = counters;
+    pl.off_o = counters + ml;
+    pl.bytes = counters + ml + o;
+    return pl;
+}
+
+static int check_decode_shape(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full) {
+    if (B < 0 || Lmax < 1 || Hq < 1 || Hkv < 1 || n_sink < 0) return SWAA_ERR_INVALID_ARG;
+    if (!is_full && window < 1) return SWAA_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || (D != 64 && D != 128)) return SWAA_ERR_UNSUPPORTED;
+    if (B > 65535) return SWAA_ERR_UNSUPPORTED;  // grid.z limit
+    return SWAA_OK;
+}
+
+}  // namespace swaa
+
+using namespace swaa;
+
+extern "C" size_t swaa_decode_workspace_size(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink,
+                                             int is_full) {
+    if (check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) != SWAA_OK || B == 0) return 256;
+    DeviceInfo info;
+    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
+    return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count).bytes;
+}
+
+extern "C" int swaa_decode_num_splits(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink,
+                                      int is_full) {
+    if (check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) != SWAA_OK || B == 0) return 1;
+    DeviceInfo info;
+    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
+    return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count).nsplit;
+}
+
+extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
+                           int B, int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full);
+    if (rc != SWAA_OK) return rc;
+    if (B == 0) return SWAA_OK;
+    if (!q || !kcache || !vcache || !out || !seqlens) return SWAA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(kcache) || !aligned16(vcache) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) != 0) return SWAA_ERR_INVALID_ARG;
+    DeviceInfo info;
+    rc = current_device_info(&info);
+    if (rc != SWAA_OK) return rc;
+    if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
+    const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < pl.bytes)
+        return SWAA_ERR_WORKSPACE;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    DecodeParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.kc = static_cast<const __nv_bfloat16*>(kcache);
+    p.vc = static_cast<const __nv_bfloat16*>(vcache);
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.seqlens = seqlens;
+    p.B = B;
+    p.Lmax = Lmax;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = Hq / Hkv;
+    p.HG = pl.HG;
+    p.window = window;
+    p.n_sink = n_sink;
+    p.is_full = is_full ? 1 : 0;
+    const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
+    p.sl2 = sc * 1.4426950408889634f;
+    p.nsplit = pl.nsplit;
+    char* ws = static_cast<char*>(workspace);
+    p.counters = reinterpret_cast<int*>(ws);
+    p.part_ml = reinterpret_cast<float*>(ws + pl.off_ml);
+    p.part_o = reinterpret_cast<float*>(ws + pl.off_o);
+    if (pl.nsplit > 1) {
+        if (cudaMemsetAsync(p.counters, 0, pl.off_ml, st) != cudaSuccess) return SWAA_ERR_CUDA;
+    }
+    const dim3 grid((unsigned)(Hkv * pl.HG), (unsigned)pl.nsplit, (unsigned)B);
+    if (D == 128) {
+        if (pl.NH == 1) decode_kernel<128, 1><<<grid, kDecodeThreads, 0, st>>>(p);
+        else decode_kernel<128, 2><<<grid, kDecodeThreads, 0, st>>>(p);
+    } else {
+        if (pl.NH == 1) decode_kernel<64, 1><<<grid, kDecodeThreads, 0, st>>>(p);
+        else decode_kernel<64, 2><<<grid, kDecodeThreads, 0, st>>>(p);
+    }
+    launch_counter().fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------- schedule
+extern "C" int swaa_schedule_is_full(const swaa_policy* policy, int layer, int phase) {
+    if (!policy || policy->n_layers < 0 || layer < 0 || layer >= policy->n_layers) return SWAA_ERR_INVALID_ARG;
+    if (phase != SWAA_PHASE_PREFILL && phase != SWAA_PHASE_DECODE) return SWAA_ERR_INVALID_ARG;
+    if (policy->fa_start < 0 || policy->fa_step < 0) return SWAA_ERR_INVALID_ARG;
+    if (phase == SWAA_PHASE_DECODE && policy->fa_decode) return 1;
+    if (policy->fa_step > 0 && layer >= policy->fa_start && (layer - policy->fa_start) % policy->fa_step == 0) return 1;
+    return 0;
+}
+
+extern "C" int swaa_schedule_fill(const swaa_policy* policy, int phase, uint8_t* is_full_out) {
+    if (!policy || !is_full_out || policy->n_layers < 0) return SWAA_ERR_INVALID_ARG;
+    for (int l = 0; l < policy->n_layers; ++l) {
+        const int r = swaa_schedule_is_full(policy, l, phase);
+        if (r < 0) return r;
+        is_full_out[l] = (uint8_t)r;
+    }
+    return SWAA_OK;
+}
+
+// ------------------------------------------------------------------------------- tile enumeration
+extern "C" int swaa_prefill_block_m(void) { return kPrefillBM; }
+extern "C" int swaa_prefill_block_n(void) { return kPrefillBN; }
+
+extern "C" int swaa_prefill_tile_range(int L, int m, int BM, int BN, int window, int n_sink, int is_full,
+                                       int* n_sink_tiles, int* n_lo, int* n_hi) {
+    if (L < 1 || BM < 1 || BN < 1 || m < 0 || (long long)m * BM >= L || n_sink < 0 || (!is_full && window < 1))
+        return SWAA_ERR_INVALID_ARG;
+    if (!n_sink_tiles || !n_lo || !n_hi) return SWAA_ERR_INVALID_ARG;
+    const int i0 = m * BM;
+    const int i1 = (L < i0 + BM ? L : i0 + BM) - 1;
+    const TileRange r = tile_range(i0, i1, BN, window, n_sink, is_full != 0);
+    *n_sink_tiles = r.n_sink_tiles;
+    *n_lo = r.n_lo;
+    *n_hi = r.n_hi;
+    return SWAA_OK;
+}
+
+extern "C" int swaa_prefill_tile_needs_mask(int L, int m, int n, int BM, int BN, int window, int n_sink,
+                                            int is_full) {
+    if (L < 1 || BM < 1 || BN < 1 || m < 0 || n < 0 || (long long)m * BM >= L || n_sink < 0 ||
+        (!is_full && window < 1))
+        return SWAA_ERR_INVALID_ARG;
+    const int i0 = m * BM;
+    const int i1 = (L < i0 + BM ? L : i0 + BM) - 1;
+    return tile_needs_mask(i0, i1, n * BN, n * BN + BN - 1, window, n_sink, is_full != 0) ? 1 : 0;
+}
+
+// ------------------------------------------------------------------------------------------ status
+extern "C" const char* swaa_status_str(int status) {
+    switch (status) {
+        case SWAA_OK: return "SWAA_OK";
+        case SWAA_ERR_INVALID_ARG: return "SWAA_ERR_INVALID_ARG";
+        case SWAA_ERR_UNSUPPORTED: return "SWAA_ERR_UNSUPPORTED";
+        case SWAA_ERR_CUDA: return "SWAA_ERR_CUDA";
+        case SWAA_ERR_WORKSPACE: return "SWAA_ERR_WORKSPACE";
+        case SWAA_ERR_BAD_SEQLENS: return "SWAA_ERR_BAD_SEQLENS";
+        case SWAA_ERR_TIMEOUT: return "SWAA_ERR_TIMEOUT";
+        default: return "SWAA_ERR_UNKNOWN";
+    }
+}
+
+extern "C" int swaa_last_device_status(void* stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SWAA_ERR_CUDA;
+    int value = 0;
+    if (cudaMemcpyFromSymbol(&value, g_device_status, sizeof(int)) != cudaSuccess) return SWAA_ERR_CUDA;
+    if (value != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return SWAA_ERR_CUDA;
+    }
+    return value;
+}
+
+extern "C" uint64_t swaa_kernel_launch_count(void) { return launch_counter().load(std::memory_order_relaxed); }
