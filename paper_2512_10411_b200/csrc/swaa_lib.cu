@@ -175,6 +175,108 @@ extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
+// ----------------------------------------------------------------------------------------- prefill
+namespace swaa {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, resolved through the runtime so that the library does not link
+// against the driver directly.
+static EncodeTiledFn encode_tiled_fn() {
+    static std::mutex mu;
+    static EncodeTiledFn fn = nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Tensor map over a token-major bf16 tensor [T, H, D]: dimensions (D, H, T) innermost first; one box is
+// [128 tokens] x [1 head] x [64 channels] = 128 rows of 128 bytes, written with the 128-byte swizzle.
+static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H, int D) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return SWAA_ERR_CUDA;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2};
+    const cuuint32_t box[3] = {64, 1, 128};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
+template <int D>
+static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const PrefillParams& p,
+                          cudaStream_t st) {
+    using L = PrefillSmem<D>;
+    if (cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
+        cudaSuccess)
+        return SWAA_ERR_CUDA;
+    const long long blocks = (long long)p.n_pairs * p.tiles_ub;
+    if (blocks > 2147483647LL) return SWAA_ERR_UNSUPPORTED;
+    prefill_kernel<D><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, p);
+    launch_counter().fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
+}  // namespace swaa
+
+extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens, int B,
+                            int T, int max_seqlen, int Hq, int Hkv, int D, int window, int n_sink, int is_full,
+                            float scale, float* lse, void* stream) {
+    if (B < 0 || T < 0 || max_seqlen < 0 || Hq < 1 || Hkv < 1 || n_sink < 0) return SWAA_ERR_INVALID_ARG;
+    if (!is_full && window < 1) return SWAA_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || (D != 64 && D != 128)) return SWAA_ERR_UNSUPPORTED;
+    if (B == 0 || T == 0) return SWAA_OK;
+    if (!q || !k || !v || !out || !cu_seqlens) return SWAA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(cu_seqlens) & 3u) != 0 || (reinterpret_cast<uintptr_t>(lse) & 3u) != 0)
+        return SWAA_ERR_INVALID_ARG;
+    DeviceInfo info;
+    int rc = current_device_info(&info);
+    if (rc != SWAA_OK) return rc;
+    if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
+
+    CUtensorMap tq, tk, tv;
+    if ((rc = make_token_major_map(&tq, q, T, Hq, D)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tk, k, T, Hkv, D)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tv, v, T, Hkv, D)) != SWAA_OK) return rc;
+
+    PrefillParams p;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.lse = lse;
+    p.cu_seqlens = cu_seqlens;
+    p.B = B;
+    p.T = T;
+    p.max_seqlen = max_seqlen;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = Hq / Hkv;
+    p.pairs_per_kv = (p.G + 1) / 2;
+    p.n_pairs = Hkv * p.pairs_per_kv;
+    const long long ub_a = (long long)T / kPrefillBM + B;
+    const long long ub_b = (long long)B * ((max_seqlen + kPrefillBM - 1) / kPrefillBM);
+    const long long ub = ub_a < ub_b ? ub_a : ub_b;
+    if (ub > 2147483647LL) return SWAA_ERR_UNSUPPORTED;
+    p.tiles_ub = (int)ub;
+    if (p.tiles_ub == 0) return SWAA_OK;  // max_seqlen == 0: nothing can be valid
+    p.window = window;
+    p.n_sink = n_sink;
+    p.is_full = is_full ? 1 : 0;
+    p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
+    p.sl2 = p.scale * 1.4426950408889634f;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return D == 128 ? launch_prefill<128>(tq, tk, tv, p, st) : launch_prefill<64>(tq, tk, tv, p, st);
+}
+
 // ---------------------------------------------------------------------------------------- schedule
 extern "C" int swaa_schedule_is_full(const swaa_policy* policy, int layer, int phase) {
     if (!policy || policy->n_layers < 0 || layer < 0 || layer >= policy->n_layers) return SWAA_ERR_INVALID_ARG;

@@ -1,7 +1,518 @@
+// Prefill attention for sm_100a: tcgen05 MMAs accumulating in tensor memory, TMA-staged operands,
+// online softmax with one thread per query row.
+//
+// Mask policy (Sec. 1, 3.1.2, 3.2.1; App. A): a query at position i of its sequence sees key j iff
+//     j <= i  and  ( is_full  or  j > i - window  or  j < n_sink ).
+// Only the key tiles that hold a visible key are visited (the sink tiles and the diagonal band), so
+// the work is O(L * window) as App. A states; the element predicate is evaluated only on tiles that
+// are not entirely visible.
+//
+// One thread block processes one 128-row query tile for TWO query heads of the same GQA group
+// ("sides" A and B).  Both sides need exactly the same K/V tiles and the same masks, so each K/V tile
+// is staged in shared memory once and feeds four MMAs.  Roles:
+//   warps 0-3   softmax of side A   (thread = query row; lane quadrant = TMEM lane quadrant)
+//   warps 4-7   softmax of side B
+//   warp  8     TMA producer (one elected lane): Q tiles once, then the K and V tile rings
+//   warp  9     MMA issuer (one elected lane) and TMEM allocation
+// Tensor memory (512 columns x 128 lanes of 32 bit): S_A | S_B | O_A | O_B.  The bf16 probabilities
+// P overwrite the first 64 columns of their own S and are consumed from TMEM as the A operand of
+// O += P V.  V tiles are used as the MN-major B operand exactly as TMA lands them.
+// Per key tile n the issuer runs  PV_A(n) QK_A(n+1) PV_B(n) QK_B(n+1), so the softmax of one side
+// overlaps the MMAs of the other.  The running maximum is only raised (and O rescaled) when it grows
+// by more than 2^8; the final division by the row sum makes the result independent of that choice.
+//
+// Every wait is bounded: a wait that runs out records SWAA_ERR_TIMEOUT, all roles leave their loops,
+// the block waits (bounded) for its outstanding copies, frees its tensor memory and returns.
 #pragma once
+
+#include <cuda.h>
+
 #include "swaa_internal.cuh"
+
 namespace swaa {
+
 constexpr int kPrefillBM = 128;
 constexpr int kPrefillBN = 128;
+constexpr int kPrefillThreads = 320;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+constexpr float kRescaleThreshold = 8.0f;                   // log2 units
+
+struct PrefillParams {
+    __nv_bfloat16* out;
+    float* lse;             // nullable, [Hq, T]
+    const int32_t* cu_seqlens;
+    int B, T, max_seqlen, Hq, Hkv, G;
+    int pairs_per_kv;       // ceil(G / 2)
+    int n_pairs;            // Hkv * pairs_per_kv
+    int tiles_ub;           // upper bound on the number of query tiles over all sequences
+    int window, n_sink, is_full;
+    float sl2;              // softmax scale * log2(e)
+    float scale;
+};
+
+// ------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-extern "C" int swaa_prefill(const void*, const void*, const void*, void*, const int32_t*, int, int, int, int, int, int, int, int, int, float, float*, void*) { return SWAA_ERR_UNSUPPORTED; }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                record_device_error(SWAA_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], "
+        "[%5];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+#define SWAA_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
+#define SWAA_I8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
+
+// 32 lanes x 32 consecutive columns: thread `lane` of the warp receives columns c .. c+31 of TMEM
+// lane (quadrant base + lane).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+        "%29,%30,%31}, [%32];"
+        : SWAA_R8(r, 0), SWAA_R8(r, 8), SWAA_R8(r, 16), SWAA_R8(r, 24)
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+        "%29,%30,%31};" ::SWAA_I8(r, 0),
+        SWAA_I8(r, 8), SWAA_I8(r, 16), SWAA_I8(r, 24), "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};" ::
+            SWAA_I8(r, 0),
+        SWAA_I8(r, 8), "r"(taddr)
+        : "memory");
+}
+
+// Shared-memory matrix descriptors for tiles stored as 128-byte rows with the 128-byte swizzle (what
+// TMA writes for a [rows][64 bf16] box).  14-bit fields hold byte values >> 4.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;  // 128-byte swizzle
+    return d;
+}
+
+// kind::f16 instruction descriptor: bf16 x bf16 -> f32, M x N, A K-major, B K- or MN-major.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+
+template <int D>
+struct PrefillSmem {
+    static constexpr int kTileBytes = 128 * D * 2;  // one 128-row tile of Q, K or V
+    static constexpr int kPanelBytes = 128 * 128;   // one [128 rows][64 ch] panel
+    static constexpr int kPanels = D / 64;
+    static constexpr int kStages = D == 128 ? 2 : 4;
+    static constexpr int kOffQ = 0;                              // two tiles (sides A, B)
+    static constexpr int kOffK = 2 * kTileBytes;                 // kStages tiles
+    static constexpr int kOffV = kOffK + kStages * kTileBytes;   // kStages tiles
+    static constexpr int kOffBar = kOffV + kStages * kTileBytes;
+    static constexpr int kNumBars = 1 + 4 * kStages + 7;
+    static constexpr int kBytes = kOffBar + kNumBars * 8 + 64;
+    static constexpr int kDynamicBytes = kBytes + 1024;          // room to align the base to 1024 B
+};
+
+template <int D>
+__global__ void __launch_bounds__(kPrefillThreads, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const PrefillParams p) {
+    using L = PrefillSmem<D>;
+    constexpr int BM = kPrefillBM, BN = kPrefillBN;
+    constexpr int ST = L::kStages;
+    constexpr uint32_t kIdescQK = make_idesc(BM, BN, 0);
+    constexpr uint32_t kIdescPV = make_idesc(BM, D, 1);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t sQ = smem_base + L::kOffQ, sK = smem_base + L::kOffK, sV = smem_base + L::kOffV;
+    const uint32_t bars = smem_base + L::kOffBar;
+    auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
+    // barrier indices
+    constexpr int BAR_Q = 0, BAR_KF = 1, BAR_KE = BAR_KF + ST, BAR_VF = BAR_KE + ST, BAR_VE = BAR_VF + ST;
+    constexpr int BAR_SF = BAR_VE + ST, BAR_PR = BAR_SF + 2, BAR_OD = BAR_PR + 2, BAR_FIN = BAR_OD + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + L::kOffBar + L::kNumBars * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* work = reinterpret_cast<int*>(tmem_slot + 2);  // {valid, start, len, m}
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- which (sequence, query tile, head pair) is this block's work item?  Heavy tiles first.
+    const int pair = blockIdx.x % p.n_pairs;
+    const int tile_id = blockIdx.x / p.n_pairs;
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        int valid = 0, w_start = 0, w_len = 0, w_m = 0;
+        int acc = 0;
+        bool bad = p.cu_seqlens[0] != 0 || p.cu_seqlens[p.B] != p.T;
+        for (int b = p.B - 1; b >= 0; --b) {  // reverse order so that the list starts with the last sequence
+            const int s = p.cu_seqlens[b], e = p.cu_seqlens[b + 1];
+            int len = e - s;
+            if (len < 0 || len > p.max_seqlen || s < 0 || e > p.T) {
+                bad = true;
+                len = 0;
+            }
+            const int nt = (len + BM - 1) / BM;
+            if (!valid && tile_id < acc + nt) {
+                valid = 1;
+                w_start = s;
+                w_len = len;
+                w_m = nt - 1 - (tile_id - acc);  // last (heaviest) tile of the sequence first
+            }
+            acc += nt;
+        }
+        if (bad) record_device_error(SWAA_ERR_BAD_SEQLENS);
+        work[0] = valid;
+        work[1] = w_start;
+        work[2] = w_len;
+        work[3] = w_m;
+        for (int i = 0; i < L::kNumBars; ++i) {
+            const bool is_pr = (i == BAR_PR || i == BAR_PR + 1);
+            mbar_init(bar(i), is_pr ? 128u : 1u);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (!work[0]) return;  // uniform: no such tile
+    const int seq_start = work[1], seq_len = work[2], m_tile = work[3];
+
+    if (warp == 9) {  // TMEM: all 512 columns (S_A, S_B, O_A, O_B)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int hk = pair / p.pairs_per_kv;
+    const int hA = hk * p.G + 2 * (pair - hk * p.pairs_per_kv);
+    const bool hasB = (hA + 1) < (hk + 1) * p.G;
+    const int i0 = m_tile * BM;
+    const int i1 = min(seq_len, i0 + BM) - 1;
+    const bool full = p.is_full != 0;
+    const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
+    const int nt = tr.count();
+
+    if (warp == 8) {
+        // =========================================================================== TMA producer
+        if (lane == 0) {
+            const int tq = seq_start + i0;
+            mbar_arrive_expect_tx(bar(BAR_Q), (hasB ? 2u : 1u) * (uint32_t)L::kTileBytes);
+#pragma unroll
+            for (int pn = 0; pn < L::kPanels; ++pn) {
+                tma_load_3d(sQ + pn * L::kPanelBytes, &tm_q, pn * 64, hA, tq, bar(BAR_Q));
+                if (hasB) tma_load_3d(sQ + L::kTileBytes + pn * L::kPanelBytes, &tm_q, pn * 64, hA + 1, tq, bar(BAR_Q));
+            }
+            bool ok = true;
+            int issued = 0;
+            for (int n = 0; n < nt && ok; ++n) {
+                const int s = n % ST;
+                const uint32_t ph = (uint32_t)(n / ST) & 1u;
+                const int tk = seq_start + tr.tile(n) * BN;
+                ok = mbar_wait(bar(BAR_KE + s), ph ^ 1u, abort_flag);
+                if (!ok) break;
+                mbar_arrive_expect_tx(bar(BAR_KF + s), (uint32_t)L::kTileBytes);
+#pragma unroll
+                for (int pn = 0; pn < L::kPanels; ++pn)
+                    tma_load_3d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, bar(BAR_KF + s));
+                ok = mbar_wait(bar(BAR_VE + s), ph ^ 1u, abort_flag);
+                if (!ok) {
+                    // the K copy just issued is still in flight: wait for it before leaving
+                    mbar_wait(bar(BAR_KF + s), ph, abort_flag);
+                    break;
+                }
+                mbar_arrive_expect_tx(bar(BAR_VF + s), (uint32_t)L::kTileBytes);
+#pragma unroll
+                for (int pn = 0; pn < L::kPanels; ++pn)
+                    tma_load_3d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, bar(BAR_VF + s));
+                issued = n + 1;
+            }
+            if (!ok) {
+                // give outstanding copies a bounded chance to land before the block's memory is released
+                const uint64_t t0 = global_timer_ns();
+                bool landed = false;
+                while (!landed && global_timer_ns() - t0 < kWaitLimitNs) {
+                    landed = mbar_try_wait(bar(BAR_Q), 0);
+                    for (int n = max(0, issued - ST); n < issued; ++n) {
+                        landed = landed && mbar_try_wait(bar(BAR_KF + n % ST), (uint32_t)(n / ST) & 1u);
+                        landed = landed && mbar_try_wait(bar(BAR_VF + n % ST), (uint32_t)(n / ST) & 1u);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 9) {
+        // ============================================================================ MMA issuer
+        if (lane == 0) {
+            const uint32_t tS[2] = {tmem_base, tmem_base + 128u};
+            const uint32_t tO[2] = {tmem_base + 256u, tmem_base + 256u + (uint32_t)D};
+            auto issue_qk = [&](int side, int stage) {
+                const uint32_t qa = sQ + side * L::kTileBytes, kb = sK + stage * L::kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (uint32_t)(kk >> 2) * L::kPanelBytes + (uint32_t)(kk & 3) * 32u;
+                    mma_ss(tS[side], smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024),
+                           kIdescQK, kk > 0 ? 1u : 0u);
+                }
+            };
+            auto issue_pv = [&](int side, int stage, bool acc) {
+                const uint32_t vb = sV + stage * L::kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk) {
+                    // P: 16 keys = 8 TMEM columns of packed bf16 pairs.  V: 16 key rows of 128 bytes.
+                    mma_ts(tO[side], tS[side] + (uint32_t)kk * 8u,
+                           smem_desc_sw128(vb + (uint32_t)kk * 2048u, L::kPanelBytes, 1024), kIdescPV,
+                           (acc || kk > 0) ? 1u : 0u);
+                }
+            };
+            bool ok = mbar_wait(bar(BAR_Q), 0, abort_flag);
+            ok = ok && mbar_wait(bar(BAR_KF + 0), 0, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0, 0);
+                tc_commit(bar(BAR_SF + 0));
+                if (hasB) {
+                    issue_qk(1, 0);
+                    tc_commit(bar(BAR_SF + 1));
+                }
+                tc_commit(bar(BAR_KE + 0));
+            }
+            for (int n = 0; n < nt && ok; ++n) {
+                const int sv = n % ST;
+                const uint32_t pv = (uint32_t)(n / ST) & 1u;
+                const bool has_next = n + 1 < nt;
+                const int sk = (n + 1) % ST;
+                const uint32_t pk = (uint32_t)((n + 1) / ST) & 1u;
+                const uint32_t pn = (uint32_t)n & 1u;
+                ok = mbar_wait(bar(BAR_PR + 0), pn, abort_flag) && mbar_wait(bar(BAR_VF + sv), pv, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(0, sv, n > 0);
+                tc_commit(bar(BAR_OD + 0));
+                if (has_next) {
+                    ok = mbar_wait(bar(BAR_KF + sk), pk, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(0, sk);
+                    tc_commit(bar(BAR_SF + 0));
+                }
+                if (hasB) {
+                    ok = mbar_wait(bar(BAR_PR + 1), pn, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(1, sv, n > 0);
+                    tc_commit(bar(BAR_OD + 1));
+                    if (has_next) {
+                        issue_qk(1, sk);
+                        tc_commit(bar(BAR_SF + 1));
+                    }
+                }
+                tc_commit(bar(BAR_VE + sv));
+                if (has_next) tc_commit(bar(BAR_KE + sk));
+            }
+            // all MMAs issued by this thread must have retired before the tensor memory is freed
+            tc_commit(bar(BAR_FIN));
+            mbar_wait(bar(BAR_FIN), 0, abort_flag);
+        }
+        __syncwarp();
+    } else {
+        // ==================================================================== softmax + epilogue
+        const int side = warp >> 2;
+        const int wq = warp & 3;
+        if (side == 0 || hasB) {
+            const int row = wq * 32 + lane;
+            const int i = i0 + row;  // position of this thread's query inside its sequence
+            const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
+            const uint32_t tS = tmem_base + lane_base + (uint32_t)side * 128u;
+            const uint32_t tO = tmem_base + lane_base + 256u + (uint32_t)side * (uint32_t)D;
+            const int h = hA + side;
+            float m_used = -INFINITY, l_sum = 0.f;
+            bool ok = true;
+            for (int n = 0; n < nt; ++n) {
+                const int j0 = tr.tile(n) * BN;
+                const bool need_mask = tile_needs_mask(i0, i1, j0, j0 + BN - 1, p.window, p.n_sink, full);
+                ok = mbar_wait(bar(BAR_SF + side), (uint32_t)n & 1u, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t sr[128];
+                tmem_ld32(tS + 0, sr + 0);
+                tmem_ld32(tS + 32, sr + 32);
+                tmem_ld32(tS + 64, sr + 64);
+                tmem_ld32(tS + 96, sr + 96);
+                tc_wait_ld();
+                if (need_mask) {
+                    const int dc = i - j0;                    // visible iff c <= dc ...
+                    const int wl = full ? -1 : dc - p.window;  // ... and ( c > wl
+                    const int sk = full ? 0 : p.n_sink - j0;   //        or c < sk )
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) {
+                        const bool vis = (c <= dc) && (c > wl || c < sk);
+                        sr[c] = vis ? sr[c] : 0xff800000u;  // -inf
+                    }
+                }
+                float rmax = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 128; ++c) rmax = fmaxf(rmax, __uint_as_float(sr[c]));
+                const float m_new = fmaxf(m_used, rmax);
+                const bool need = (m_used != -INFINITY) && ((m_new - m_used) * p.sl2 > kRescaleThreshold);
+                if (__any_sync(0xffffffffu, need)) {
+                    // raise the reference maximum of every row of this warp and rescale O accordingly
+                    ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(n - 1) & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const float alpha = (m_used == -INFINITY) ? 1.f : ex2f((m_used - m_new) * p.sl2);
+#pragma unroll
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t orr[32];
+                        tmem_ld32(tO + cc * 32, orr);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                        tmem_st32(tO + cc * 32, orr);
+                    }
+                    tc_wait_st();
+                    l_sum *= alpha;
+                    m_used = m_new;
+                } else if (m_used == -INFINITY) {
+                    m_used = m_new;  // nothing accumulated yet for this row
+                }
+                const float off = (m_used == -INFINITY) ? 0.f : m_used * p.sl2;
+                float psum = 0.f;
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const float p0 = ex2f(fmaf(__uint_as_float(sr[cc * 32 + 2 * c]), p.sl2, -off));
+                        const float p1 = ex2f(fmaf(__uint_as_float(sr[cc * 32 + 2 * c + 1]), p.sl2, -off));
+                        psum += p0 + p1;
+                        pk[c] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(tS + cc * 16, pk);
+                }
+                l_sum += psum;
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(BAR_PR + side));
+            }
+            if (ok) ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(nt - 1) & 1u, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+                const bool row_valid = i < seq_len;
+                __nv_bfloat16* orow = p.out + ((size_t)(seq_start + i) * p.Hq + h) * D;
+#pragma unroll
+                for (int cc = 0; cc < D / 32; ++cc) {
+                    uint32_t orr[32];
+                    tmem_ld32(tO + cc * 32, orr);
+                    tc_wait_ld();
+                    if (row_valid) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(orr[v * 8 + 0]) * inv, __uint_as_float(orr[v * 8 + 1]) * inv);
+                            w.y = pack_bf16x2(__uint_as_float(orr[v * 8 + 2]) * inv, __uint_as_float(orr[v * 8 + 3]) * inv);
+                            w.z = pack_bf16x2(__uint_as_float(orr[v * 8 + 4]) * inv, __uint_as_float(orr[v * 8 + 5]) * inv);
+                            w.w = pack_bf16x2(__uint_as_float(orr[v * 8 + 6]) * inv, __uint_as_float(orr[v * 8 + 7]) * inv);
+                            *reinterpret_cast<uint4*>(orow + cc * 32 + v * 8) = w;
+                        }
+                    }
+                }
+                if (row_valid && p.lse != nullptr) {
+                    const float lse2 = (m_used == -INFINITY) ? -INFINITY : m_used * p.sl2 + log2f(l_sum);
+                    p.lse[(size_t)h * p.T + seq_start + i] = lse2 * 0.6931471805599453f;
+                }
+            }
+        }
+    }
+
+    // ---- teardown: every thread arrives here (also after a failed wait); free the tensor memory
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace swaa

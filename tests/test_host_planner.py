@@ -1,0 +1,122 @@
+"""CPU tests of the host-side logic of the library: tile enumeration, layer schedule, symbol table.
+
+The tile enumeration is the part of the prefill kernel that makes work linear in L (App. A); expanded to
+(query, key) pairs on the CPU it must cover the oracle's visible set exactly, and tiles reported as
+needing no mask must be entirely visible.
+"""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2512_10411_b200 as swaa
+from paper_2512_10411_b200.build import build_library
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build_library()
+    return swaa.load_library()
+
+
+def test_library_exports_every_declared_symbol(_lib):
+    with open(os.path.join(ROOT, "include", "swaa.h")) as f:
+        text = f.read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = set(re.findall(r"\b(swaa_[a-z0-9_]+)\s*\(", text))
+    assert {"swaa_prefill", "swaa_decode", "swaa_decode_workspace_size", "swaa_schedule_is_full",
+            "swaa_schedule_fill", "swaa_status_str", "swaa_last_device_status"} <= names
+    for n in sorted(names):
+        assert hasattr(_lib, n), f"libswaa.so does not export {n}"
+
+
+def _visible_matrix(L, W, S, full):
+    return np.array([[oracle.visible(i, j, W, S, full) for j in range(L)] for i in range(L)], dtype=bool)
+
+
+CASES = [(L, W, S, full) for L in (1, 5, 16, 17, 40, 67) for W in (1, 3, 8, 20, 100) for S in (0, 1, 7, 30)
+         for full in (False, True) if not (full and (W, S) != (1, 0))]
+
+
+@pytest.mark.parametrize("BM,BN", [(8, 8), (16, 4), (4, 16), (7, 5)])
+def test_tile_enumeration_covers_exactly_the_visible_set(BM, BN):
+    for L, W, S, full in CASES:
+        vis = _visible_matrix(L, W, S, full)
+        covered = np.zeros_like(vis)
+        for m in range((L + BM - 1) // BM):
+            ns, lo, hi = swaa.prefill_tile_range(L, m, BM, BN, W, S, full)
+            tiles = list(range(ns)) + list(range(lo, hi + 1))
+            assert len(set(tiles)) == len(tiles), "a tile is visited twice"
+            i0, i1 = m * BM, min(L, (m + 1) * BM)
+            for n in tiles:
+                j0, j1 = n * BN, min(L, (n + 1) * BN)
+                block = vis[i0:i1, j0:j1]
+                assert block.any(), f"tile without a visible pair: {(L, W, S, full, m, n)}"
+                if not swaa.prefill_tile_needs_mask(L, m, n, BM, BN, W, S, full):
+                    assert block.all() and (n + 1) * BN <= L, (L, W, S, full, m, n)
+                covered[i0:i1, j0:j1] = True
+        assert not (vis & ~covered).any(), f"visible pair outside the enumerated tiles: {(L, W, S, full)}"
+
+
+def test_tile_counts_of_the_benchmark_workloads():
+    """Tiles visited per head at the kernel's own tile shape: linear in L for SWA, quadratic for full."""
+    BM, BN = swaa.prefill_block_shape()
+    assert (BM, BN) == (128, 128)
+
+    def count(L, W, S, full):
+        total = 0
+        for m in range((L + BM - 1) // BM):
+            ns, lo, hi = swaa.prefill_tile_range(L, m, BM, BN, W, S, full)
+            total += ns + hi - lo + 1
+        return total
+
+    assert count(1024, 128, 4, False) == 21
+    assert count(32768, 2048, 4, False) == 4455
+    assert count(32768, 1, 0, True) == 32896
+    a, b = count(32768, 2048, 4, False), count(65536, 2048, 4, False)
+    assert b - a == 256 * 18  # each further query tile costs 16 band tiles + diagonal + sink tile
+
+
+def test_schedule_matches_paper_patterns():
+    golden = os.path.join(ROOT, "tests", "golden", "fa_layer_patterns.txt")
+    with open(golden) as f:
+        rows = [ln for ln in f if ln.strip() and not ln.startswith("#")]
+    for ln in rows:
+        name, start, step, first, count = [x.strip() for x in ln.split(";")]
+        pol = swaa.SwaaPolicy(36, 2048, 10, int(start), int(step), False)
+        fa = [l for l, f_ in enumerate(swaa.schedule_fill(pol, 0)) if f_]
+        assert len(fa) == int(count) and fa[: len(first.split())] == [int(x) for x in first.split()], name
+        for phase in (0, 1):
+            for fa_decode in (False, True):
+                pol = swaa.SwaaPolicy(36, 2048, 10, int(start), int(step), fa_decode)
+                got = swaa.schedule_fill(pol, phase)
+                want = [oracle.layer_is_full(l, int(start), int(step), fa_decode, phase) for l in range(36)]
+                assert got == want
+                assert [swaa.schedule_is_full(pol, l, phase) for l in range(36)] == want
+
+
+def test_schedule_argument_errors():
+    pol = swaa.SwaaPolicy(4, 8, 0, 1, 2, False)
+    for layer, phase in ((-1, 0), (4, 0), (0, 2)):
+        with pytest.raises(swaa.SwaaError):
+            swaa.schedule_is_full(pol, layer, phase)
+    with pytest.raises(swaa.SwaaError):
+        swaa.schedule_fill(swaa.SwaaPolicy(4, 8, 0, -1, 2, False), 0)
+
+
+def test_status_strings():
+    assert swaa.status_str(0) == "SWAA_OK"
+    assert swaa.status_str(-6) == "SWAA_ERR_TIMEOUT"
+    assert swaa.status_str(-99) == "SWAA_ERR_UNKNOWN"
+
+
+def test_decode_split_plan_is_consistent():
+    for args in ((16, 32, 8, 128, 65536, 4096, 4, 1), (16, 32, 8, 128, 65536, 4096, 4, 0), (1, 4, 2, 64, 100, 8, 0, 0)):
+        ns = swaa.decode_num_splits(*args)
+        assert ns >= 1
+        B, Hq, Hkv, D = args[:4]
+        assert swaa.decode_workspace_size(*args) >= B * Hq * ns * (D + 2) * 4
