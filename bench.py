@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the SWAA attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+    layer schedule (host)  ->  swaa_prefill on the long-context SWA workload (L=32768, Hq=32, Hkv=8,
+    D=128, W=2048, n_sink=4)  ->  swaa_decode with full attention ("FA Decode") on the decode workload
+    (B=16, 65536-entry cache)  ->  swaa_decode with the SWA mask (n_sink=4 + W=4096 entries).
+Each kernel is bracketed by CUDA events on the launching stream; L2 is flushed (256 MiB write) before
+each kernel so every launch reads its inputs from HBM.  `value` is the effective prefill throughput
+4*D*Hq*visible_pairs / (prefill kernel time), aggregated over ranks (max time over ranks); decode
+bandwidth goes into the `decode` object.  With N > 1 every rank runs the same independent problem
+(weak scaling, no collective on the data path).
+
+--impl reference times the float64 CPU oracle (the only "reference" this method has) on a bounded
+row sample of the same prefill workload, on the host cores, rank 0 only.
+"""
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "swa_prefill_effective_tflops"
+UNIT = "TFLOP/s"
+L2_FLUSH_BYTES = 256 << 20
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
+# summarised under profiles/ (None until a capture exists).
+PREFILL_DRAM_TRAFFIC_BYTES = None
+
+
+def visible_pairs(L, W, S, full):
+    if full or W >= L:
+        return L * (L + 1) // 2
+    if L >= W + S:
+        return W * (W + 1) // 2 + (L - W) * W + S * (S + 1) // 2 + (L - W - S) * S
+    return sum(min(i + 1, W) + max(0, min(S, i - W + 1)) for i in range(L))
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, uuid: str, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._uuid, self._period = uuid, period_s
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if isinstance(uuid, str) else uuid)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self._period)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def run_reference(args, rank):
+    """The oracle as it stands, on the host cores: each step computes a bounded row sample of the
+    long-context SWA prefill workload; throughput is reported in the same unit as the GPU arm."""
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+    from paper_2512_10411_b200 import inputs
+
+    cfg = inputs.cfg_long()
+    q, k, v, cu = inputs.make_prefill_inputs(cfg, "cpu")
+    qh, kh, vh = (inputs.to_f32_numpy(t) for t in (q, k, v))
+    L = cfg.seqlens[0]
+    rng = np.random.default_rng(1234)
+
+    def sample(n):
+        rt = rng.integers(cfg.window + cfg.n_sink, L, n)  # rows with a full window: S + W visible keys each
+        rh = rng.integers(0, cfg.Hq, n).astype(np.int32)
+        return rt, rh
+
+    def run(rows):
+        t0 = time.perf_counter()
+        r = oracle.prefill(qh, kh, vh, [0, L], cfg.window, cfg.n_sink, False, rows=rows)
+        dt = time.perf_counter() - t0
+        return dt, 4.0 * cfg.D * float(r["nvis"].sum())
+
+    dt, _ = run(sample(256))
+    budget = 150.0 / max(1, args.steps + args.warmup)          # whole run within a few minutes
+    n_rows = int(max(32, min(65536, 256 * min(budget, 20.0) / max(dt, 1e-6))))
+    for _ in range(args.warmup):
+        run(sample(n_rows))
+    total_t, total_f = 0.0, 0.0
+    for _ in range(args.steps):
+        dt, fl = run(sample(n_rows))
+        total_t += dt
+        total_f += fl
+    value = total_f / total_t / 1e12
+    cores = oracle.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg2 long-context SWA prefill: B=1 L=32768 Hq=32 Hkv=8 D=128 W=2048 n_sink=4",
+                   "sample": f"{n_rows} seeded (row, head) rows per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{n_rows} seeded (row, head) rows per step, {args.steps} steps"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args, rank, local_rank, world):
+    import numpy as np
+    import torch
+
+    import paper_2512_10411_b200 as swaa
+    from paper_2512_10411_b200 import inputs
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    swaa.load_library()
+    peaks = load_peaks()
+
+    # ---------------------------------------------------------------- workloads (resident in HBM)
+    pcfg = inputs.cfg_long()
+    q, k, v, cu = inputs.make_prefill_inputs(pcfg, dev)
+    out = torch.empty_like(q)
+    L = pcfg.seqlens[0]
+    dcfg = inputs.cfg_decode()
+    dq, kc, vc, sl = inputs.make_decode_inputs(dcfg, dev)
+    dout = torch.empty_like(dq)
+    ws_fa = torch.empty(swaa.decode_workspace_size(dcfg.B, dcfg.Hq, dcfg.Hkv, dcfg.D, dcfg.Lmax, dcfg.window,
+                                                   dcfg.n_sink, True), dtype=torch.uint8, device=dev)
+    ws_swa = torch.empty(swaa.decode_workspace_size(dcfg.B, dcfg.Hq, dcfg.Hkv, dcfg.D, dcfg.Lmax, dcfg.window,
+                                                    dcfg.n_sink, False), dtype=torch.uint8, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    # one SWAA recipe: SWA prefill on this layer, FA decode on; and its SWA-decode counterpart
+    pol_fa_decode = swaa.SwaaPolicy(n_layers=36, window=pcfg.window, n_sink=pcfg.n_sink, fa_start=3, fa_step=4,
+                                    fa_decode=True)
+    pol_swa_decode = swaa.SwaaPolicy(n_layers=36, window=dcfg.window, n_sink=dcfg.n_sink, fa_start=3, fa_step=4,
+                                     fa_decode=False)
+    layer = 0
+
+    prefill_flops = 4.0 * pcfg.D * pcfg.Hq * visible_pairs(L, pcfg.window, pcfg.n_sink, False)
+    fa_bytes = float(dcfg.B) * dcfg.Lmax * dcfg.Hkv * dcfg.D * 2 * 2
+    swa_bytes = float(dcfg.B) * (dcfg.window + dcfg.n_sink) * dcfg.Hkv * dcfg.D * 2 * 2
+    stream = torch.cuda.current_stream()
+
+    def step(events=None):
+        full_p = swaa.schedule_is_full(pol_fa_decode, layer, 0)
+        full_d = swaa.schedule_is_full(pol_fa_decode, layer, 1)
+        full_s = swaa.schedule_is_full(pol_swa_decode, layer, 1)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)] if events is not None else None
+        flush.zero_()
+        if ev: ev[0].record(stream)
+        swaa.swaa_prefill(q, k, v, out, cu, L, pcfg.window, pcfg.n_sink, full_p)
+        if ev: ev[1].record(stream)
+        flush.zero_()
+        if ev: ev[2].record(stream)
+        swaa.swaa_decode(dq, kc, vc, dout, sl, dcfg.window, dcfg.n_sink, full_d, ws_fa)
+        if ev: ev[3].record(stream)
+        flush.zero_()
+        if ev: ev[4].record(stream)
+        swaa.swaa_decode(dq, kc, vc, dout, sl, dcfg.window, dcfg.n_sink, full_s, ws_swa)
+        if ev: ev[5].record(stream)
+        if events is not None:
+            events.append(ev)
+        return full_p, full_d, full_s
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        flags = step()
+    assert flags == (False, True, False)
+    barrier()
+    assert swaa.last_device_status() == 0
+
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    launches0 = swaa.kernel_launch_count()
+    events = []
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    t_start.record(stream)
+    for _ in range(args.steps):
+        step(events)
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = swaa.kernel_launch_count() - launches0
+    assert swaa.last_device_status() == 0
+    total_ms = t_start.elapsed_time(t_end)
+    t_pre = sum(e[0].elapsed_time(e[1]) for e in events)
+    t_fa = sum(e[2].elapsed_time(e[3]) for e in events)
+    t_swa = sum(e[4].elapsed_time(e[5]) for e in events)
+
+    # ---------------------------------------------------------------- end to end from host buffers
+    qh, kh, vh = (t.cpu().pin_memory() for t in (q, k, v))
+    outh = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    dqh, douth = dq.cpu().pin_memory(), torch.empty(dout.shape, dtype=dout.dtype).pin_memory()
+    q2, k2, v2, dq2 = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v), torch.empty_like(dq)
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        q2.copy_(qh, non_blocking=True)
+        k2.copy_(kh, non_blocking=True)
+        v2.copy_(vh, non_blocking=True)
+        swaa.swaa_prefill(q2, k2, v2, out, cu, L, pcfg.window, pcfg.n_sink, False)
+        outh.copy_(out, non_blocking=True)
+
+    def e2e_decode_step(full, ws):
+        dq2.copy_(dqh, non_blocking=True)
+        swaa.swaa_decode(dq2, kc, vc, dout, sl, dcfg.window, dcfg.n_sink, full, ws)
+        douth.copy_(dout, non_blocking=True)
+
+    def time_loop(fn, n):
+        fn()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n):
+            fn()
+        b.record(stream)
+        barrier()
+        return a.elapsed_time(b) / n
+
+    e2e_ms = time_loop(e2e_step, e2e_steps)
+    e2e_fa_ms = time_loop(lambda: e2e_decode_step(True, ws_fa), e2e_steps)
+    e2e_swa_ms = time_loop(lambda: e2e_decode_step(False, ws_swa), e2e_steps)
+
+    # ---------------------------------------------------------------- max over ranks
+    times = torch.tensor([total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms = times.tolist()
+    K, N = args.steps, world
+
+    cpu_baseline = None
+    if rank == 0 and N == 1:
+        import oracle
+
+        qf, kf, vf = (inputs.to_f32_numpy(t) for t in (q, k, v))
+        rng = np.random.default_rng(1234)
+
+        def oracle_rows(n):
+            rt = rng.integers(pcfg.window + pcfg.n_sink, L, n)
+            rh = rng.integers(0, pcfg.Hq, n).astype(np.int32)
+            t0 = time.perf_counter()
+            r = oracle.prefill(qf, kf, vf, [0, L], pcfg.window, pcfg.n_sink, False, rows=(rt, rh))
+            return time.perf_counter() - t0, 4.0 * pcfg.D * float(r["nvis"].sum())
+
+        dt, _ = oracle_rows(512)
+        n_rows = int(max(512, min(1 << 20, 512 * 15.0 / max(dt, 1e-6))))  # about 15 s of CPU work
+        dt, fl = oracle_rows(n_rows)
+        cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": f"{n_rows} seeded (row, head) rows of the same workload, {dt:.1f} s"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    avg_pre_ms = t_pre / K
+    achieved = prefill_flops / (avg_pre_ms * 1e-3) / 1e12
+    fa_gbs = fa_bytes / (t_fa / K * 1e-3) / 1e9
+    swa_gbs = swa_bytes / (t_swa / K * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": N * achieved, "unit": UNIT, "n_gpus": N, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "cfg2 long-context SWA prefill: B=1 L=32768 Hq=32 Hkv=8 D=128 W=2048 n_sink=4 "
+                               "(K row 0 shifted); step also runs cfg4 decode B=16 Lcache=65536 FA and SWA(W=4096,n_sink=4)",
+                   "l2": "flushed by a 256 MiB write before every kernel", "parallelism": f"replicas x{N}",
+                   "value_from": "prefill kernel time inside the step (CUDA events on the launching stream)"},
+        "clocks": clocks,
+        "e2e": {"value": N * prefill_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                "h2d_bytes_per_step": int(q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": int(out.numel()) * 2,
+                "ms_per_step": e2e_ms},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "prefill_kernel<128>", "bound": "tensor", "achieved": achieved,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                     "traffic": PREFILL_DRAM_TRAFFIC_BYTES, "peak_source": peaks["source"] + " burst bf16",
+                     "frac_of_nominal_2250": achieved / 2250.0, "ms_per_launch": avg_pre_ms},
+        "decode": {
+            "fa": {"gbs": N * fa_gbs, "us_per_launch": 1e3 * t_fa / K, "bytes": fa_bytes,
+                   "roofline": {"bound": "hbm", "achieved": fa_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                "frac": fa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": fa_gbs / 8000.0},
+                   "e2e_gbs": fa_bytes / (e2e_fa_ms * 1e-3) / 1e9},
+            "swa": {"gbs": N * swa_gbs, "us_per_launch": 1e3 * t_swa / K, "bytes": swa_bytes,
+                    "roofline": {"bound": "hbm", "achieved": swa_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                 "frac": swa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": swa_gbs / 8000.0},
+                    "e2e_gbs": swa_bytes / (e2e_swa_ms * 1e-3) / 1e9},
+        },
+        "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()
