@@ -97,6 +97,33 @@ int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out
                 size_t workspace_bytes, void* stream);
 
 /*
+ * Allocation-free decode.  (The paper has no counterpart to this call; it exists for integration.)
+ *
+ * Same computation and arguments as swaa_decode, but the split-K scratch lives in a fixed array inside
+ * the library's device image, so the caller passes no workspace and nothing is allocated, by this
+ * call or on its behalf.  It is meant for callers that cannot call cudaMalloc at the point where
+ * attention runs: code on a latency-critical serving path, where an allocation would stall the whole
+ * device; a plug-in that receives tensors from a host framework but has no handle on that framework's
+ * memory pool, and must not take memory behind its back; a process whose device memory is already
+ * handed out in full to other owners.
+ *
+ *   - The scratch array is SWAA_DECODE_STATIC_SCRATCH_BYTES (16 MiB) per GPU, held by every GPU that
+ *     loads the library until the process exits.  A shape whose scratch need
+ *     (swaa_decode_workspace_size) exceeds it is rejected with SWAA_ERR_WORKSPACE and nothing runs;
+ *     use swaa_decode with a caller-owned workspace for those.
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current) before it launches.  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call left
+ *     there; each call clears the part that must start at zero.  Two calls whose kernels can overlap
+ *     on the same GPU (different streams, no dependency between them) race on it: serialise them.
+ * Returns the same status codes as swaa_decode.
+ */
+#define SWAA_DECODE_STATIC_SCRATCH_BYTES (16u << 20)
+int swaa_decode_static(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
+                       int B, int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
+                       void* stream);
+
+/*
  * Layer schedule (host only).  Sec. 3.1.2: a fixed-interval subset of layers keeps full attention
  * (Table 1 "FA layers": [1,3,5,...], [0,2,4,...], [1,5,9,...], [1,9,17,...], [3,7,11,...]); Sec. 3.1.1:
  * with FA decode every layer is full while decoding.  Layers are 0-based.

@@ -68,6 +68,8 @@ def load_library():
     lib.swaa_decode_num_splits.restype = ci
     lib.swaa_decode.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
     lib.swaa_decode.restype = ci
+    lib.swaa_decode_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp]
+    lib.swaa_decode_static.restype = ci
     lib.swaa_schedule_is_full.argtypes = [ctypes.POINTER(_Policy), ci, ci]
     lib.swaa_schedule_is_full.restype = ci
     lib.swaa_schedule_fill.argtypes = [ctypes.POINTER(_Policy), ci, ctypes.POINTER(ctypes.c_uint8)]
@@ -157,6 +159,28 @@ def swaa_decode(q, kcache, vcache, out, seqlens, window: int, n_sink: int, is_fu
                          _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_decode")
+
+
+DECODE_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def swaa_decode_static(q, kcache, vcache, out, seqlens, window: int, n_sink: int, is_full: bool, scale: float = 0.0,
+                       stream=None) -> None:
+    """Forwards to C swaa_decode_static: decode with the library's built-in scratch array, for callers
+    that cannot allocate a workspace.  Shapes whose scratch need exceeds DECODE_STATIC_SCRATCH_BYTES raise
+    SwaaError(SWAA_ERR_WORKSPACE).  Calls on one GPU share the array: do not let two overlap."""
+    lib = load_library()
+    B, Hq, D = q.shape
+    _, Lmax, Hkv, _ = kcache.shape
+    if tuple(kcache.shape) != (B, Lmax, Hkv, D) or tuple(vcache.shape) != (B, Lmax, Hkv, D) \
+            or tuple(out.shape) != (B, Hq, D) or seqlens.numel() != B:
+        raise ValueError("swaa_decode_static: inconsistent tensor shapes")
+    bf = torch.bfloat16
+    rc = lib.swaa_decode_static(_dev_ptr(q, bf, "q"), _dev_ptr(kcache, bf, "kcache"), _dev_ptr(vcache, bf, "vcache"),
+                                _dev_ptr(out, bf, "out"), _dev_ptr(seqlens, torch.int32, "seqlens"), B, Lmax, Hq, Hkv,
+                                D, int(window), int(n_sink), int(bool(is_full)), float(scale), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_decode_static")
 
 
 def schedule_is_full(policy: SwaaPolicy, layer: int, phase: int) -> bool:

@@ -277,6 +277,53 @@ extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* o
     return D == 128 ? launch_prefill<128>(tq, tk, tv, p, st) : launch_prefill<64>(tq, tk, tv, p, st);
 }
 
+// ------------------------------------------------------------------- decode without allocation
+namespace swaa {
+
+// Split-K scratch of swaa_decode_static.  One instance per device that loads this module; shared by
+// every call on that device.  In host code this name is only a handle for cudaGetSymbolAddress: it
+// is not a device address and must never be handed to a kernel.
+static __device__ __align__(256) unsigned char g_decode_static_scratch[SWAA_DECODE_STATIC_SCRATCH_BYTES];
+
+// Device address of the scratch array on the current device, looked up once per device.
+static int decode_static_scratch(void** out) {
+    static std::mutex mu;
+    static void* table[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SWAA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (table[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_decode_static_scratch) != cudaSuccess || ptr == nullptr) {
+            (void)cudaGetLastError();
+            return SWAA_ERR_CUDA;
+        }
+        table[dev] = ptr;
+    }
+    *out = table[dev];
+    return SWAA_OK;
+}
+
+}  // namespace swaa
+
+extern "C" int swaa_decode_static(const void* q, const void* kcache, const void* vcache, void* out,
+                                  const int32_t* seqlens, int B, int Lmax, int Hq, int Hkv, int D, int window,
+                                  int n_sink, int is_full, float scale, void* stream) {
+    const int rc = check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full);
+    if (rc != SWAA_OK) return rc;
+    if (B == 0) return SWAA_OK;
+    // Reject what does not fit the fixed array before touching the device.
+    if (swaa_decode_workspace_size(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) > SWAA_DECODE_STATIC_SCRATCH_BYTES)
+        return SWAA_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    const int rs = decode_static_scratch(&scratch);
+    if (rs != SWAA_OK) return rs;
+    // Same kernel and same plan as swaa_decode; its ticket counters (the only part that must start at
+    // zero) are cleared by that call on `stream` before the kernel runs.
+    return swaa_decode(q, kcache, vcache, out, seqlens, B, Lmax, Hq, Hkv, D, window, n_sink, is_full, scale, scratch,
+                       SWAA_DECODE_STATIC_SCRATCH_BYTES, stream);
+}
+
 // ---------------------------------------------------------------------------------------- schedule
 extern "C" int swaa_schedule_is_full(const swaa_policy* policy, int layer, int phase) {
     if (!policy || policy->n_layers < 0 || layer < 0 || layer >= policy->n_layers) return SWAA_ERR_INVALID_ARG;
