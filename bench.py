@@ -357,13 +357,49 @@ def run_ours(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
+def run_profile_case(case: str):
+    """A few launches of one kernel on its benchmark workload and nothing else: the command that the
+    ncu captures summarised under profiles/ run."""
+    import torch
+
+    import paper_2512_10411_b200 as swaa
+    from paper_2512_10411_b200 import inputs
+
+    torch.cuda.set_device(0)
+    if case.startswith("prefill"):
+        cfg = {"prefill": inputs.cfg_long(), "prefill_full": inputs.cfg_long(is_full=True),
+               "prefill_tiny": inputs.cfg_tiny()}[case]
+        q, k, v, cu = inputs.make_prefill_inputs(cfg, "cuda")
+        out = torch.empty_like(q)
+        for _ in range(3):
+            swaa.swaa_prefill(q, k, v, out, cu, cfg.seqlens[0], cfg.window, cfg.n_sink, cfg.is_full)
+    else:
+        cfg = inputs.cfg_decode(B=4) if case.endswith("_small") else inputs.cfg_decode()
+        full = "fa" in case
+        q, kc, vc, sl = inputs.make_decode_inputs(cfg, "cuda")
+        ws = torch.empty(swaa.decode_workspace_size(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.Lmax, cfg.window, cfg.n_sink,
+                                                    full), dtype=torch.uint8, device="cuda")
+        out = torch.empty_like(q)
+        for _ in range(3):
+            swaa.swaa_decode(q, kc, vc, out, sl, cfg.window, cfg.n_sink, full, ws)
+    assert swaa.last_device_status() == 0
+    print(json.dumps({"profile_case": case, "launches": swaa.kernel_launch_count()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--profile-case", default=None,
+                    choices=["prefill", "prefill_full", "prefill_tiny", "decode_fa", "decode_swa", "decode_fa_small",
+                             "decode_swa_small"],
+                    help="run three launches of one kernel only (for ncu) and exit")
     args = ap.parse_args()
+    if args.profile_case:
+        run_profile_case(args.profile_case)
+        return
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -33,7 +33,7 @@ namespace swaa {
 
 constexpr int kPrefillBM = 128;
 constexpr int kPrefillBN = 128;
-constexpr int kPrefillThreads = 320;
+constexpr int kPrefillThreads = 384;  // 8 softmax warps + 4 auxiliary warps (producer, issuer, 2 idle)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 constexpr float kRescaleThreshold = 8.0f;                   // log2 units
 
@@ -124,6 +124,31 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
         "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+
+// Packed pairs of fp32 in one 64-bit register (two lanes per FMA/ADD instruction on sm_100).
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 #define SWAA_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
@@ -273,7 +298,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
     const int nt = tr.count();
 
-    if (warp == 8) {
+    // Register budget per scheduler partition: two softmax warps at 216 + one auxiliary warp at 72.
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+      if (warp == 8) {
         // =========================================================================== TMA producer
         if (lane == 0) {
             const int tq = seq_start + i0;
@@ -321,7 +349,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
         }
         __syncwarp();
-    } else if (warp == 9) {
+      } else if (warp == 9) {
         // ============================================================================ MMA issuer
         if (lane == 0) {
             const uint32_t tS[2] = {tmem_base, tmem_base + 128u};
@@ -395,8 +423,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mbar_wait(bar(BAR_FIN), 0, abort_flag);
         }
         __syncwarp();
+      }
     } else {
         // ==================================================================== softmax + epilogue
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         const int side = warp >> 2;
         const int wq = warp & 3;
         if (side == 0 || hasB) {
@@ -430,9 +460,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         sr[c] = vis ? sr[c] : 0xff800000u;  // -inf
                     }
                 }
-                float rmax = -INFINITY;
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < 128; ++c) rmax = fmaxf(rmax, __uint_as_float(sr[c]));
+                for (int c = 0; c < 128; c += 8) {
+                    mx0 = fmax3(mx0, __uint_as_float(sr[c + 0]), __uint_as_float(sr[c + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+                    mx2 = fmax3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+                    mx3 = fmax3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
+                }
+                const float rmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                 const float m_new = fmaxf(m_used, rmax);
                 const bool need = (m_used != -INFINITY) && ((m_new - m_used) * p.sl2 > kRescaleThreshold);
                 if (__any_sync(0xffffffffu, need)) {
@@ -457,20 +493,30 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     m_used = m_new;  // nothing accumulated yet for this row
                 }
                 const float off = (m_used == -INFINITY) ? 0.f : m_used * p.sl2;
-                float psum = 0.f;
+                const uint64_t sl2x2 = pack_f32x2(p.sl2, p.sl2), noffx2 = pack_f32x2(-off, -off);
+                uint64_t psum_a = pack_f32x2(0.f, 0.f), psum_b = pack_f32x2(0.f, 0.f);
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
-                        const float p0 = ex2f(fmaf(__uint_as_float(sr[cc * 32 + 2 * c]), p.sl2, -off));
-                        const float p1 = ex2f(fmaf(__uint_as_float(sr[cc * 32 + 2 * c + 1]), p.sl2, -off));
-                        psum += p0 + p1;
+                        const uint64_t x = fma_f32x2(
+                            pack_f32x2(__uint_as_float(sr[cc * 32 + 2 * c]), __uint_as_float(sr[cc * 32 + 2 * c + 1])),
+                            sl2x2, noffx2);
+                        float x0, x1;
+                        unpack_f32x2(x, x0, x1);
+                        const float p0 = ex2f(x0), p1 = ex2f(x1);
+                        if (c & 1) psum_b = add_f32x2(psum_b, pack_f32x2(p0, p1));
+                        else psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
                         pk[c] = pack_bf16x2(p0, p1);
                     }
                     tmem_st16(tS + cc * 16, pk);
                 }
-                l_sum += psum;
+                {
+                    float a0, a1;
+                    unpack_f32x2(add_f32x2(psum_a, psum_b), a0, a1);
+                    l_sum += a0 + a1;
+                }
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(BAR_PR + side));
