@@ -398,4 +398,15 @@ extern "C" int swaa_last_device_status(void* stream) {
     return value;
 }
 
+#ifdef SWAA_PHASE_TIMING
+extern "C" int swaa_debug_read_phases(unsigned long long* out32, int reset) {
+    if (cudaMemcpyFromSymbol(out32, g_phase_cycles, sizeof(unsigned long long) * 32) != cudaSuccess) return SWAA_ERR_CUDA;
+    if (reset) {
+        unsigned long long z[32] = {0};
+        if (cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z)) != cudaSuccess) return SWAA_ERR_CUDA;
+    }
+    return SWAA_OK;
+}
+#endif
+
 extern "C" uint64_t swaa_kernel_launch_count(void) { return launch_counter().load(std::memory_order_relaxed); }

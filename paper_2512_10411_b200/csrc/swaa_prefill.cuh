@@ -199,6 +199,17 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int b_mn_major) 
            ((uint32_t)(M >> 4) << 24);
 }
 
+#ifdef SWAA_PHASE_TIMING
+// Development aid: per-phase cycle sums of the softmax role (side A: 0-7, side B: 8-15) and of the
+// issuer's waits (16-23), accumulated over all blocks.
+__device__ unsigned long long g_phase_cycles[32];
+#define SWAA_TICK(var) const long long var = clock64()
+#define SWAA_PHASE_ADD(slot, cycles) atomicAdd(&g_phase_cycles[slot], (unsigned long long)(cycles))
+#else
+#define SWAA_TICK(var)
+#define SWAA_PHASE_ADD(slot, cycles)
+#endif
+
 template <int D>
 struct PrefillSmem {
     static constexpr int kTileBytes = 128 * D * 2;  // one 128-row tile of Q, K or V
@@ -441,23 +452,35 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (int n = 0; n < nt; ++n) {
                 const int j0 = tr.tile(n) * BN;
                 const bool need_mask = tile_needs_mask(i0, i1, j0, j0 + BN - 1, p.window, p.n_sink, full);
+                SWAA_TICK(c0);
                 ok = mbar_wait(bar(BAR_SF + side), (uint32_t)n & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
+                SWAA_TICK(c1);
                 uint32_t sr[128];
                 tmem_ld32(tS + 0, sr + 0);
                 tmem_ld32(tS + 32, sr + 32);
                 tmem_ld32(tS + 64, sr + 64);
                 tmem_ld32(tS + 96, sr + 96);
                 tc_wait_ld();
+                SWAA_TICK(c2);
+                uint32_t vis[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
                 if (need_mask) {
-                    const int dc = i - j0;                    // visible iff c <= dc ...
-                    const int wl = full ? -1 : dc - p.window;  // ... and ( c > wl
-                    const int sk = full ? 0 : p.n_sink - j0;   //        or c < sk )
+                    // Bit b of vis[cc] <=> column c = 32*cc + b of this tile is visible to this row:
+                    //   c <= dc  and  ( c > wl  or  c < sk ).
+                    const int dc = i - j0;
+                    const int wl = full ? -1 : dc - p.window;
+                    const int sk = full ? 0 : p.n_sink - j0;
 #pragma unroll
-                    for (int c = 0; c < 128; ++c) {
-                        const bool vis = (c <= dc) && (c > wl || c < sk);
-                        sr[c] = vis ? sr[c] : 0xff800000u;  // -inf
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const int d = dc - 32 * cc, w = wl - 32 * cc, sn = sk - 32 * cc;
+                        const uint32_t causal = d >= 31 ? 0xffffffffu : (d < 0 ? 0u : ((2u << d) - 1u));
+                        const uint32_t win = w < 0 ? 0xffffffffu : (w >= 31 ? 0u : ~((2u << w) - 1u));
+                        const uint32_t snk = sn <= 0 ? 0u : (sn >= 32 ? 0xffffffffu : ((1u << sn) - 1u));
+                        vis[cc] = causal & (win | snk);
+#pragma unroll
+                        for (int b = 0; b < 32; ++b)
+                            sr[cc * 32 + b] = ((vis[cc] >> b) & 1u) ? sr[cc * 32 + b] : 0xff800000u;  // -inf
                     }
                 }
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -492,12 +515,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 } else if (m_used == -INFINITY) {
                     m_used = m_new;  // nothing accumulated yet for this row
                 }
+                SWAA_TICK(c3);
                 const float off = (m_used == -INFINITY) ? 0.f : m_used * p.sl2;
                 const uint64_t sl2x2 = pack_f32x2(p.sl2, p.sl2), noffx2 = pack_f32x2(-off, -off);
                 uint64_t psum_a = pack_f32x2(0.f, 0.f), psum_b = pack_f32x2(0.f, 0.f);
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     uint32_t pk[16];
+                    if (need_mask && __all_sync(0xffffffffu, vis[cc] == 0u)) {
+                        // no row of this warp sees any of these 32 keys: P = 0 without touching the MUFU
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                        tmem_st16(tS + cc * 16, pk);
+                        continue;
+                    }
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
                         const uint64_t x = fma_f32x2(
@@ -517,9 +548,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     unpack_f32x2(add_f32x2(psum_a, psum_b), a0, a1);
                     l_sum += a0 + a1;
                 }
+                SWAA_TICK(c4);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(BAR_PR + side));
+#ifdef SWAA_PHASE_TIMING
+                if (lane == 0 && wq == 0) {
+                    const long long c5 = clock64();
+                    SWAA_PHASE_ADD(side * 8 + 0, c1 - c0);  // wait for S
+                    SWAA_PHASE_ADD(side * 8 + 1, c2 - c1);  // TMEM load
+                    SWAA_PHASE_ADD(side * 8 + 2, c3 - c2);  // mask + max (+ rescale)
+                    SWAA_PHASE_ADD(side * 8 + 3, c4 - c3);  // exp, pack, store issue
+                    SWAA_PHASE_ADD(side * 8 + 4, c5 - c4);  // store wait + arrive
+                    SWAA_PHASE_ADD(side * 8 + 5, 1);        // tiles
+                }
+#endif
             }
             if (ok) ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(nt - 1) & 1u, abort_flag);
             if (ok) {
