@@ -215,13 +215,14 @@ static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H
 
 template <int D>
 static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const PrefillParams& p,
-                          cudaStream_t st) {
+                          int sm_count, cudaStream_t st) {
     using L = PrefillSmem<D>;
     if (cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
         cudaSuccess)
         return SWAA_ERR_CUDA;
-    const long long blocks = (long long)p.n_pairs * p.tiles_ub;
-    if (blocks > 2147483647LL) return SWAA_ERR_UNSUPPORTED;
+    // persistent blocks: one per SM (or fewer when there is less work), each walks its share of the items
+    long long blocks = (long long)p.n_pairs * p.tiles_ub;
+    if (blocks > sm_count) blocks = sm_count;
     prefill_kernel<D><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
@@ -265,7 +266,7 @@ extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* o
     const long long ub_a = (long long)T / kPrefillBM + B;
     const long long ub_b = (long long)B * ((max_seqlen + kPrefillBM - 1) / kPrefillBM);
     const long long ub = ub_a < ub_b ? ub_a : ub_b;
-    if (ub > 2147483647LL) return SWAA_ERR_UNSUPPORTED;
+    if (ub > 2147483647LL / p.n_pairs) return SWAA_ERR_UNSUPPORTED;
     p.tiles_ub = (int)ub;
     if (p.tiles_ub == 0) return SWAA_OK;  // max_seqlen == 0: nothing can be valid
     p.window = window;
@@ -274,7 +275,8 @@ extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* o
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
     p.sl2 = p.scale * 1.4426950408889634f;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return D == 128 ? launch_prefill<128>(tq, tk, tv, p, st) : launch_prefill<64>(tq, tk, tv, p, st);
+    return D == 128 ? launch_prefill<128>(tq, tk, tv, p, info.sm_count, st)
+                    : launch_prefill<64>(tq, tk, tv, p, info.sm_count, st);
 }
 
 // ------------------------------------------------------------------- decode without allocation

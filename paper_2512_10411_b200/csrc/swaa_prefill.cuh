@@ -220,9 +220,17 @@ struct PrefillSmem {
     static constexpr int kOffK = 2 * kTileBytes;                 // kStages tiles
     static constexpr int kOffV = kOffK + kStages * kTileBytes;   // kStages tiles
     static constexpr int kOffBar = kOffV + kStages * kTileBytes;
-    static constexpr int kNumBars = 1 + 4 * kStages + 7;
-    static constexpr int kBytes = kOffBar + kNumBars * 8 + 64;
+    // barriers: Q full/empty, K full/empty, V full/empty per stage, per side S-full / P-ready / O-done /
+    // O-free, work-descriptor full/empty per slot, final
+    static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1;
+    static constexpr int kOffMisc = kOffBar + kNumBars * 8;      // tmem slot, abort flag, work descriptors
+    static constexpr int kBytes = kOffMisc + 128;
     static constexpr int kDynamicBytes = kBytes + 1024;          // room to align the base to 1024 B
+};
+
+// One unit of work: a 128-row query tile of one sequence for one pair of query heads.
+struct WorkItem {
+    int valid, seq_start, seq_len, m_tile, pair;
 };
 
 template <int D>
@@ -242,53 +250,27 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t bars = smem_base + L::kOffBar;
     auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
     // barrier indices
-    constexpr int BAR_Q = 0, BAR_KF = 1, BAR_KE = BAR_KF + ST, BAR_VF = BAR_KE + ST, BAR_VE = BAR_VF + ST;
-    constexpr int BAR_SF = BAR_VE + ST, BAR_PR = BAR_SF + 2, BAR_OD = BAR_PR + 2, BAR_FIN = BAR_OD + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + L::kOffBar + L::kNumBars * 8);
+    constexpr int BAR_QF = 0, BAR_QE = 1, BAR_KF = 2, BAR_KE = BAR_KF + ST, BAR_VF = BAR_KE + ST, BAR_VE = BAR_VF + ST;
+    constexpr int BAR_SF = BAR_VE + ST, BAR_PR = BAR_SF + 2, BAR_OD = BAR_PR + 2, BAR_OF = BAR_OD + 2;
+    constexpr int BAR_WF = BAR_OF + 2, BAR_WE = BAR_WF + 2, BAR_FIN = BAR_WE + 2;
+    static_assert(BAR_FIN + 1 == L::kNumBars, "barrier count");
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + L::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    int* work = reinterpret_cast<int*>(tmem_slot + 2);  // {valid, start, len, m}
+    volatile int* work_ring = reinterpret_cast<volatile int*>(tmem_slot + 4);  // 2 slots x 8 ints
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool full = p.is_full != 0;
 
-    // ---- which (sequence, query tile, head pair) is this block's work item?  Heavy tiles first.
-    const int pair = blockIdx.x % p.n_pairs;
-    const int tile_id = blockIdx.x / p.n_pairs;
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        int valid = 0, w_start = 0, w_len = 0, w_m = 0;
-        int acc = 0;
-        bool bad = p.cu_seqlens[0] != 0 || p.cu_seqlens[p.B] != p.T;
-        for (int b = p.B - 1; b >= 0; --b) {  // reverse order so that the list starts with the last sequence
-            const int s = p.cu_seqlens[b], e = p.cu_seqlens[b + 1];
-            int len = e - s;
-            if (len < 0 || len > p.max_seqlen || s < 0 || e > p.T) {
-                bad = true;
-                len = 0;
-            }
-            const int nt = (len + BM - 1) / BM;
-            if (!valid && tile_id < acc + nt) {
-                valid = 1;
-                w_start = s;
-                w_len = len;
-                w_m = nt - 1 - (tile_id - acc);  // last (heaviest) tile of the sequence first
-            }
-            acc += nt;
-        }
-        if (bad) record_device_error(SWAA_ERR_BAD_SEQLENS);
-        work[0] = valid;
-        work[1] = w_start;
-        work[2] = w_len;
-        work[3] = w_m;
         for (int i = 0; i < L::kNumBars; ++i) {
-            const bool is_pr = (i == BAR_PR || i == BAR_PR + 1);
-            mbar_init(bar(i), is_pr ? 128u : 1u);
+            uint32_t count = 1u;
+            if (i == BAR_PR || i == BAR_PR + 1 || i == BAR_OF || i == BAR_OF + 1) count = 128u;  // softmax threads
+            if (i == BAR_WE || i == BAR_WE + 1) count = 10u;  // producer, issuer, one lane per softmax warp
+            mbar_init(bar(i), count);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
-    if (!work[0]) return;  // uniform: no such tile
-    const int seq_start = work[1], seq_len = work[2], m_tile = work[3];
-
     if (warp == 9) {  // TMEM: all 512 columns (S_A, S_B, O_A, O_B)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(512u)
@@ -300,59 +282,122 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int hk = pair / p.pairs_per_kv;
-    const int hA = hk * p.G + 2 * (pair - hk * p.pairs_per_kv);
-    const bool hasB = (hA + 1) < (hk + 1) * p.G;
-    const int i0 = m_tile * BM;
-    const int i1 = min(seq_len, i0 + BM) - 1;
-    const bool full = p.is_full != 0;
-    const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
-    const int nt = tr.count();
+    // Consumers of the work ring: wait for descriptor `it`, copy it, release the slot.
+    auto fetch_work = [&](int it, WorkItem& w, bool release) -> bool {
+        const int slot = it & 1;
+        if (!mbar_wait(bar(BAR_WF + slot), (uint32_t)(it >> 1) & 1u, abort_flag)) return false;
+        volatile int* d = work_ring + slot * 8;
+        w.valid = d[0];
+        w.seq_start = d[1];
+        w.seq_len = d[2];
+        w.m_tile = d[3];
+        w.pair = d[4];
+        if (release) mbar_arrive(bar(BAR_WE + slot));
+        return true;
+    };
 
     // Register budget per scheduler partition: two softmax warps at 216 + one auxiliary warp at 72.
     if (warp >= 8) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-      if (warp == 8) {
+      if (warp == 10) {
+        // ====================================================================== work scheduler
+        // Walks this block's work items w = blockIdx.x, blockIdx.x + gridDim.x, ... and publishes their
+        // descriptors.  Items are ordered heavy-first: last sequence first, last tile of a sequence first.
+        if (lane == 0) {
+            if (p.cu_seqlens[0] != 0 || p.cu_seqlens[p.B] != p.T) record_device_error(SWAA_ERR_BAD_SEQLENS);
+            int b = p.B, acc = 0, cur_nt = 0, cur_s = 0, cur_len = 0;
+            auto next_seq = [&]() {
+                acc += cur_nt;
+                --b;
+                cur_nt = 0;
+                if (b >= 0) {
+                    const int s0 = p.cu_seqlens[b], e0 = p.cu_seqlens[b + 1];
+                    int len = e0 - s0;
+                    if (len < 0 || len > p.max_seqlen || s0 < 0 || e0 > p.T) {
+                        record_device_error(SWAA_ERR_BAD_SEQLENS);
+                        len = 0;
+                    }
+                    cur_s = s0;
+                    cur_len = len;
+                    cur_nt = (len + BM - 1) / BM;
+                }
+            };
+            next_seq();
+            for (int it = 0;; ++it) {
+                const long long w = (long long)blockIdx.x + (long long)it * gridDim.x;
+                const long long tile_id = w / p.n_pairs;
+                const int pair = (int)(w - tile_id * p.n_pairs);
+                while (b >= 0 && tile_id >= (long long)acc + cur_nt) next_seq();
+                const int slot = it & 1;
+                if (!mbar_wait(bar(BAR_WE + slot), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag)) break;
+                volatile int* d = work_ring + slot * 8;
+                d[0] = b >= 0 ? 1 : 0;
+                d[1] = cur_s;
+                d[2] = cur_len;
+                d[3] = b >= 0 ? cur_nt - 1 - (int)(tile_id - acc) : 0;
+                d[4] = pair;
+                mbar_arrive(bar(BAR_WF + slot));
+                if (b < 0) break;
+            }
+        }
+        __syncwarp();
+      } else if (warp == 8) {
         // =========================================================================== TMA producer
         if (lane == 0) {
-            const int tq = seq_start + i0;
-            mbar_arrive_expect_tx(bar(BAR_Q), (hasB ? 2u : 1u) * (uint32_t)L::kTileBytes);
-#pragma unroll
-            for (int pn = 0; pn < L::kPanels; ++pn) {
-                tma_load_3d(sQ + pn * L::kPanelBytes, &tm_q, pn * 64, hA, tq, bar(BAR_Q));
-                if (hasB) tma_load_3d(sQ + L::kTileBytes + pn * L::kPanelBytes, &tm_q, pn * 64, hA + 1, tq, bar(BAR_Q));
-            }
-            bool ok = true;
-            int issued = 0;
-            for (int n = 0; n < nt && ok; ++n) {
-                const int s = n % ST;
-                const uint32_t ph = (uint32_t)(n / ST) & 1u;
-                const int tk = seq_start + tr.tile(n) * BN;
-                ok = mbar_wait(bar(BAR_KE + s), ph ^ 1u, abort_flag);
+            int g = 0;           // K/V tiles issued so far (ring position)
+            bool ok = true, q_in_flight = false;
+            int items = 0;
+            for (int it = 0; ok; ++it) {
+                WorkItem w;
+                ok = fetch_work(it, w, true);
+                if (!ok || !w.valid) break;
+                const int hk = w.pair / p.pairs_per_kv;
+                const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
+                const bool hasB = (hA + 1) < (hk + 1) * p.G;
+                const int i0 = w.m_tile * BM, i1 = min(w.seq_len, i0 + BM) - 1;
+                const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
+                const int nt = tr.count();
+                // Q tiles of both sides (the previous item's last QK must have retired)
+                ok = mbar_wait(bar(BAR_QE), ((uint32_t)items & 1u) ^ 1u, abort_flag);
                 if (!ok) break;
-                mbar_arrive_expect_tx(bar(BAR_KF + s), (uint32_t)L::kTileBytes);
+                const int tq = w.seq_start + i0;
+                mbar_arrive_expect_tx(bar(BAR_QF), (hasB ? 2u : 1u) * (uint32_t)L::kTileBytes);
 #pragma unroll
-                for (int pn = 0; pn < L::kPanels; ++pn)
-                    tma_load_3d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, bar(BAR_KF + s));
-                ok = mbar_wait(bar(BAR_VE + s), ph ^ 1u, abort_flag);
-                if (!ok) {
-                    // the K copy just issued is still in flight: wait for it before leaving
-                    mbar_wait(bar(BAR_KF + s), ph, abort_flag);
-                    break;
+                for (int pn = 0; pn < L::kPanels; ++pn) {
+                    tma_load_3d(sQ + pn * L::kPanelBytes, &tm_q, pn * 64, hA, tq, bar(BAR_QF));
+                    if (hasB)
+                        tma_load_3d(sQ + L::kTileBytes + pn * L::kPanelBytes, &tm_q, pn * 64, hA + 1, tq, bar(BAR_QF));
                 }
-                mbar_arrive_expect_tx(bar(BAR_VF + s), (uint32_t)L::kTileBytes);
+                q_in_flight = true;
+                ++items;
+                for (int n = 0; n < nt; ++n, ++g) {
+                    const int s = g % ST;
+                    const uint32_t ph = (uint32_t)(g / ST) & 1u;
+                    const int tk = w.seq_start + tr.tile(n) * BN;
+                    ok = mbar_wait(bar(BAR_KE + s), ph ^ 1u, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(bar(BAR_KF + s), (uint32_t)L::kTileBytes);
 #pragma unroll
-                for (int pn = 0; pn < L::kPanels; ++pn)
-                    tma_load_3d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, bar(BAR_VF + s));
-                issued = n + 1;
+                    for (int pn = 0; pn < L::kPanels; ++pn)
+                        tma_load_3d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, bar(BAR_KF + s));
+                    ok = mbar_wait(bar(BAR_VE + s), ph ^ 1u, abort_flag);
+                    if (!ok) {
+                        mbar_wait(bar(BAR_KF + s), ph, abort_flag);  // the K copy just issued
+                        break;
+                    }
+                    mbar_arrive_expect_tx(bar(BAR_VF + s), (uint32_t)L::kTileBytes);
+#pragma unroll
+                    for (int pn = 0; pn < L::kPanels; ++pn)
+                        tma_load_3d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, bar(BAR_VF + s));
+                }
             }
             if (!ok) {
                 // give outstanding copies a bounded chance to land before the block's memory is released
                 const uint64_t t0 = global_timer_ns();
                 bool landed = false;
                 while (!landed && global_timer_ns() - t0 < kWaitLimitNs) {
-                    landed = mbar_try_wait(bar(BAR_Q), 0);
-                    for (int n = max(0, issued - ST); n < issued; ++n) {
+                    landed = !q_in_flight || mbar_try_wait(bar(BAR_QF), (uint32_t)(items - 1) & 1u);
+                    for (int n = max(0, g - ST); n < g; ++n) {
                         landed = landed && mbar_try_wait(bar(BAR_KF + n % ST), (uint32_t)(n / ST) & 1u);
                         landed = landed && mbar_try_wait(bar(BAR_VF + n % ST), (uint32_t)(n / ST) & 1u);
                     }
@@ -384,50 +429,77 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                            (acc || kk > 0) ? 1u : 0u);
                 }
             };
-            bool ok = mbar_wait(bar(BAR_Q), 0, abort_flag);
-            ok = ok && mbar_wait(bar(BAR_KF + 0), 0, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                issue_qk(0, 0);
-                tc_commit(bar(BAR_SF + 0));
-                if (hasB) {
-                    issue_qk(1, 0);
-                    tc_commit(bar(BAR_SF + 1));
-                }
-                tc_commit(bar(BAR_KE + 0));
-            }
-            for (int n = 0; n < nt && ok; ++n) {
-                const int sv = n % ST;
-                const uint32_t pv = (uint32_t)(n / ST) & 1u;
-                const bool has_next = n + 1 < nt;
-                const int sk = (n + 1) % ST;
-                const uint32_t pk = (uint32_t)((n + 1) / ST) & 1u;
-                const uint32_t pn = (uint32_t)n & 1u;
-                ok = mbar_wait(bar(BAR_PR + 0), pn, abort_flag) && mbar_wait(bar(BAR_VF + sv), pv, abort_flag);
+            int g = 0;                 // K/V ring position
+            int gs[2] = {0, 0};        // tiles processed per side (phase of S-full / P-ready / O-done)
+            int items_side[2] = {0, 0};
+            int items = 0;
+            bool ok = true;
+            for (int it = 0; ok; ++it) {
+                WorkItem w;
+                ok = fetch_work(it, w, true);
+                if (!ok || !w.valid) break;
+                const int hk = w.pair / p.pairs_per_kv;
+                const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
+                const bool hasB = (hA + 1) < (hk + 1) * p.G;
+                const int i0 = w.m_tile * BM, i1 = min(w.seq_len, i0 + BM) - 1;
+                const int nt = tile_range(i0, i1, BN, p.window, p.n_sink, full).count();
+                ok = mbar_wait(bar(BAR_QF), (uint32_t)items & 1u, abort_flag) &&
+                     mbar_wait(bar(BAR_KF + g % ST), (uint32_t)(g / ST) & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_pv(0, sv, n > 0);
-                tc_commit(bar(BAR_OD + 0));
-                if (has_next) {
-                    ok = mbar_wait(bar(BAR_KF + sk), pk, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(0, sk);
-                    tc_commit(bar(BAR_SF + 0));
-                }
+                issue_qk(0, g % ST);
+                tc_commit(bar(BAR_SF + 0));
                 if (hasB) {
-                    ok = mbar_wait(bar(BAR_PR + 1), pn, abort_flag);
+                    issue_qk(1, g % ST);
+                    tc_commit(bar(BAR_SF + 1));
+                }
+                tc_commit(bar(BAR_KE + g % ST));
+                if (nt == 1) tc_commit(bar(BAR_QE));  // Q is no longer needed by this item
+                for (int n = 0; n < nt; ++n, ++g) {
+                    const int sv = g % ST;
+                    const uint32_t pv = (uint32_t)(g / ST) & 1u;
+                    const bool has_next = n + 1 < nt;
+                    const int sk = (g + 1) % ST;
+                    const uint32_t pk = (uint32_t)((g + 1) / ST) & 1u;
+                    ok = mbar_wait(bar(BAR_PR + 0), (uint32_t)gs[0] & 1u, abort_flag) &&
+                         mbar_wait(bar(BAR_VF + sv), pv, abort_flag);
+                    // the first PV of an item overwrites O: the previous item's epilogue must have read it
+                    if (ok && n == 0) ok = mbar_wait(bar(BAR_OF + 0), ((uint32_t)items_side[0] & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(1, sv, n > 0);
-                    tc_commit(bar(BAR_OD + 1));
+                    issue_pv(0, sv, n > 0);
+                    tc_commit(bar(BAR_OD + 0));
+                    ++gs[0];
                     if (has_next) {
-                        issue_qk(1, sk);
-                        tc_commit(bar(BAR_SF + 1));
+                        ok = mbar_wait(bar(BAR_KF + sk), pk, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_qk(0, sk);
+                        tc_commit(bar(BAR_SF + 0));
+                    }
+                    if (hasB) {
+                        ok = mbar_wait(bar(BAR_PR + 1), (uint32_t)gs[1] & 1u, abort_flag);
+                        if (ok && n == 0)
+                            ok = mbar_wait(bar(BAR_OF + 1), ((uint32_t)items_side[1] & 1u) ^ 1u, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(1, sv, n > 0);
+                        tc_commit(bar(BAR_OD + 1));
+                        ++gs[1];
+                        if (has_next) {
+                            issue_qk(1, sk);
+                            tc_commit(bar(BAR_SF + 1));
+                        }
+                    }
+                    tc_commit(bar(BAR_VE + sv));
+                    if (has_next) {
+                        tc_commit(bar(BAR_KE + sk));
+                        if (n + 2 == nt) tc_commit(bar(BAR_QE));  // that was the item's last QK
                     }
                 }
-                tc_commit(bar(BAR_VE + sv));
-                if (has_next) tc_commit(bar(BAR_KE + sk));
+                ++items;
+                ++items_side[0];
+                if (hasB) ++items_side[1];
             }
             // all MMAs issued by this thread must have retired before the tensor memory is freed
             tc_commit(bar(BAR_FIN));
@@ -440,20 +512,35 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         const int side = warp >> 2;
         const int wq = warp & 3;
-        if (side == 0 || hasB) {
-            const int row = wq * 32 + lane;
+        const int row = wq * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
+        const uint32_t tS = tmem_base + lane_base + (uint32_t)side * 128u;
+        const uint32_t tO = tmem_base + lane_base + 256u + (uint32_t)side * (uint32_t)D;
+        int gs = 0;  // tiles processed by this side so far
+        bool ok = true;
+        for (int it = 0; ok; ++it) {
+            WorkItem w;
+            ok = fetch_work(it, w, false);
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_WE + (it & 1)));
+            if (!w.valid) break;
+            const int hk = w.pair / p.pairs_per_kv;
+            const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
+            const bool hasB = (hA + 1) < (hk + 1) * p.G;
+            if (side == 1 && !hasB) continue;
+            const int seq_start = w.seq_start, seq_len = w.seq_len;
+            const int i0 = w.m_tile * BM, i1 = min(seq_len, i0 + BM) - 1;
+            const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
+            const int nt = tr.count();
             const int i = i0 + row;  // position of this thread's query inside its sequence
-            const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
-            const uint32_t tS = tmem_base + lane_base + (uint32_t)side * 128u;
-            const uint32_t tO = tmem_base + lane_base + 256u + (uint32_t)side * (uint32_t)D;
             const int h = hA + side;
             float m_used = -INFINITY, l_sum = 0.f;
-            bool ok = true;
-            for (int n = 0; n < nt; ++n) {
+            for (int n = 0; n < nt; ++n, ++gs) {
                 const int j0 = tr.tile(n) * BN;
                 const bool need_mask = tile_needs_mask(i0, i1, j0, j0 + BN - 1, p.window, p.n_sink, full);
                 SWAA_TICK(c0);
-                ok = mbar_wait(bar(BAR_SF + side), (uint32_t)n & 1u, abort_flag);
+                ok = mbar_wait(bar(BAR_SF + side), (uint32_t)gs & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 SWAA_TICK(c1);
@@ -473,9 +560,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const int sk = full ? 0 : p.n_sink - j0;
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
-                        const int d = dc - 32 * cc, w = wl - 32 * cc, sn = sk - 32 * cc;
+                        const int d = dc - 32 * cc, wd = wl - 32 * cc, sn = sk - 32 * cc;
                         const uint32_t causal = d >= 31 ? 0xffffffffu : (d < 0 ? 0u : ((2u << d) - 1u));
-                        const uint32_t win = w < 0 ? 0xffffffffu : (w >= 31 ? 0u : ~((2u << w) - 1u));
+                        const uint32_t win = wd < 0 ? 0xffffffffu : (wd >= 31 ? 0u : ~((2u << wd) - 1u));
                         const uint32_t snk = sn <= 0 ? 0u : (sn >= 32 ? 0xffffffffu : ((1u << sn) - 1u));
                         vis[cc] = causal & (win | snk);
 #pragma unroll
@@ -496,7 +583,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const bool need = (m_used != -INFINITY) && ((m_new - m_used) * p.sl2 > kRescaleThreshold);
                 if (__any_sync(0xffffffffu, need)) {
                     // raise the reference maximum of every row of this warp and rescale O accordingly
-                    ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(n - 1) & 1u, abort_flag);
+                    ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(gs - 1) & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     const float alpha = (m_used == -INFINITY) ? 1.f : ex2f((m_used - m_new) * p.sl2);
@@ -564,34 +651,44 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
 #endif
             }
-            if (ok) ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(nt - 1) & 1u, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-                const bool row_valid = i < seq_len;
+            if (!ok) break;
+            // ---- epilogue of this item: O / l -> bf16 -> global
+            SWAA_TICK(e0);
+            ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(gs - 1) & 1u, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t orr[D];
+#pragma unroll
+            for (int cc = 0; cc < D / 32; ++cc) tmem_ld32(tO + cc * 32, orr + cc * 32);
+            tc_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar(BAR_OF + side));  // O may be overwritten by the next item's first PV
+            SWAA_TICK(e1);
+            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            if (i < seq_len) {
                 __nv_bfloat16* orow = p.out + ((size_t)(seq_start + i) * p.Hq + h) * D;
 #pragma unroll
-                for (int cc = 0; cc < D / 32; ++cc) {
-                    uint32_t orr[32];
-                    tmem_ld32(tO + cc * 32, orr);
-                    tc_wait_ld();
-                    if (row_valid) {
-#pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(orr[v * 8 + 0]) * inv, __uint_as_float(orr[v * 8 + 1]) * inv);
-                            w.y = pack_bf16x2(__uint_as_float(orr[v * 8 + 2]) * inv, __uint_as_float(orr[v * 8 + 3]) * inv);
-                            w.z = pack_bf16x2(__uint_as_float(orr[v * 8 + 4]) * inv, __uint_as_float(orr[v * 8 + 5]) * inv);
-                            w.w = pack_bf16x2(__uint_as_float(orr[v * 8 + 6]) * inv, __uint_as_float(orr[v * 8 + 7]) * inv);
-                            *reinterpret_cast<uint4*>(orow + cc * 32 + v * 8) = w;
-                        }
-                    }
+                for (int v = 0; v < D / 8; ++v) {
+                    uint4 o4;
+                    o4.x = pack_bf16x2(__uint_as_float(orr[v * 8 + 0]) * inv, __uint_as_float(orr[v * 8 + 1]) * inv);
+                    o4.y = pack_bf16x2(__uint_as_float(orr[v * 8 + 2]) * inv, __uint_as_float(orr[v * 8 + 3]) * inv);
+                    o4.z = pack_bf16x2(__uint_as_float(orr[v * 8 + 4]) * inv, __uint_as_float(orr[v * 8 + 5]) * inv);
+                    o4.w = pack_bf16x2(__uint_as_float(orr[v * 8 + 6]) * inv, __uint_as_float(orr[v * 8 + 7]) * inv);
+                    *reinterpret_cast<uint4*>(orow + v * 8) = o4;
                 }
-                if (row_valid && p.lse != nullptr) {
+                if (p.lse != nullptr) {
                     const float lse2 = (m_used == -INFINITY) ? -INFINITY : m_used * p.sl2 + log2f(l_sum);
                     p.lse[(size_t)h * p.T + seq_start + i] = lse2 * 0.6931471805599453f;
                 }
             }
+#ifdef SWAA_PHASE_TIMING
+            if (lane == 0 && wq == 0) {
+                const long long e2 = clock64();
+                SWAA_PHASE_ADD(side * 8 + 6, e1 - e0);  // epilogue: wait + O load
+                SWAA_PHASE_ADD(side * 8 + 7, e2 - e1);  // epilogue: convert + store
+                SWAA_PHASE_ADD(16 + side, 1);           // items
+            }
+#endif
         }
     }
 
