@@ -200,12 +200,12 @@ static EncodeTiledFn encode_tiled_fn() {
 
 // Tensor map over a token-major bf16 tensor [T, H, D]: dimensions (D, H, T) innermost first; one box is
 // [128 tokens] x [1 head] x [64 channels] = 128 rows of 128 bytes, written with the 128-byte swizzle.
-static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H, int D) {
+static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H, int D, int box_tokens = 128) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return SWAA_ERR_CUDA;
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T};
     const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2};
-    const cuuint32_t box[3] = {64, 1, 128};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)box_tokens};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -214,8 +214,8 @@ static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H
 }
 
 template <int D>
-static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const PrefillParams& p,
-                          int sm_count, cudaStream_t st) {
+static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                          const PrefillParams& p, int sm_count, cudaStream_t st) {
     using L = PrefillSmem<D>;
     if (cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
         cudaSuccess)
@@ -223,7 +223,7 @@ static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CU
     // persistent blocks: one per SM (or fewer when there is less work), each walks its share of the items
     long long blocks = (long long)p.n_pairs * p.tiles_ub;
     if (blocks > sm_count) blocks = sm_count;
-    prefill_kernel<D><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, p);
+    prefill_kernel<D><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
@@ -246,10 +246,11 @@ extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* o
     if (rc != SWAA_OK) return rc;
     if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     if ((rc = make_token_major_map(&tq, q, T, Hq, D)) != SWAA_OK) return rc;
     if ((rc = make_token_major_map(&tk, k, T, Hkv, D)) != SWAA_OK) return rc;
     if ((rc = make_token_major_map(&tv, v, T, Hkv, D)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&to, out, T, Hq, D, 32)) != SWAA_OK) return rc;  // output rows, 32 at a time
 
     PrefillParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
@@ -275,8 +276,8 @@ extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* o
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
     p.sl2 = p.scale * 1.4426950408889634f;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return D == 128 ? launch_prefill<128>(tq, tk, tv, p, info.sm_count, st)
-                    : launch_prefill<64>(tq, tk, tv, p, info.sm_count, st);
+    return D == 128 ? launch_prefill<128>(tq, tk, tv, to, p, info.sm_count, st)
+                    : launch_prefill<64>(tq, tk, tv, to, p, info.sm_count, st);
 }
 
 // ------------------------------------------------------------------- decode without allocation

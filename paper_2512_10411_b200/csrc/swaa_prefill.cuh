@@ -99,6 +99,21 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// Store of one box from shared memory (bulk async-group completion).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -219,7 +234,8 @@ struct PrefillSmem {
     static constexpr int kOffQ = 0;                              // two tiles (sides A, B)
     static constexpr int kOffK = 2 * kTileBytes;                 // kStages tiles
     static constexpr int kOffV = kOffK + kStages * kTileBytes;   // kStages tiles
-    static constexpr int kOffBar = kOffV + kStages * kTileBytes;
+    static constexpr int kOffStage = kOffV + kStages * kTileBytes;  // 8 x 4 KiB: per-warp output staging
+    static constexpr int kOffBar = kOffStage + 8 * 4096;
     // barriers: Q full/empty, K full/empty, V full/empty per stage, per side S-full / P-ready / O-done /
     // O-free, work-descriptor full/empty per slot, final
     static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1;
@@ -236,7 +252,8 @@ struct WorkItem {
 template <int D>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-               const __grid_constant__ CUtensorMap tm_v, const PrefillParams p) {
+               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+               const PrefillParams p) {
     using L = PrefillSmem<D>;
     constexpr int BM = kPrefillBM, BN = kPrefillBN;
     constexpr int ST = L::kStages;
@@ -247,6 +264,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t sQ = smem_base + L::kOffQ, sK = smem_base + L::kOffK, sV = smem_base + L::kOffV;
+    const uint32_t sStage = smem_base + L::kOffStage;
     const uint32_t bars = smem_base + L::kOffBar;
     auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
     // barrier indices
@@ -665,7 +683,32 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mbar_arrive(bar(BAR_OF + side));  // O may be overwritten by the next item's first PV
             SWAA_TICK(e1);
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            if (i < seq_len) {
+            if (i0 + wq * 32 + 31 < seq_len) {
+                // all 32 rows of this warp are valid: stage [32 rows][64 ch] panels in shared memory in the
+                // 128-byte-swizzled layout and let TMA write them (fully coalesced, off the LSU path)
+                const uint32_t stage = sStage + (uint32_t)warp * 4096u;
+#pragma unroll
+                for (int pn = 0; pn < D / 64; ++pn) {
+                    if (lane == 0) tma_store_wait_read();  // the previous store has finished reading the stage
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t* o8 = orr + pn * 64 + j * 8;
+                        st_shared_v4(stage + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) * 16),
+                                     pack_bf16x2(__uint_as_float(o8[0]) * inv, __uint_as_float(o8[1]) * inv),
+                                     pack_bf16x2(__uint_as_float(o8[2]) * inv, __uint_as_float(o8[3]) * inv),
+                                     pack_bf16x2(__uint_as_float(o8[4]) * inv, __uint_as_float(o8[5]) * inv),
+                                     pack_bf16x2(__uint_as_float(o8[6]) * inv, __uint_as_float(o8[7]) * inv));
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_3d(&tm_o, stage, pn * 64, h, seq_start + i0 + wq * 32);
+                        tma_store_commit();
+                    }
+                }
+            } else if (i < seq_len) {
+                // ragged tail of a sequence: plain predicated row stores
                 __nv_bfloat16* orow = p.out + ((size_t)(seq_start + i) * p.Hq + h) * D;
 #pragma unroll
                 for (int v = 0; v < D / 8; ++v) {
@@ -676,10 +719,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     o4.w = pack_bf16x2(__uint_as_float(orr[v * 8 + 6]) * inv, __uint_as_float(orr[v * 8 + 7]) * inv);
                     *reinterpret_cast<uint4*>(orow + v * 8) = o4;
                 }
-                if (p.lse != nullptr) {
-                    const float lse2 = (m_used == -INFINITY) ? -INFINITY : m_used * p.sl2 + log2f(l_sum);
-                    p.lse[(size_t)h * p.T + seq_start + i] = lse2 * 0.6931471805599453f;
-                }
+            }
+            if (i < seq_len && p.lse != nullptr) {
+                const float lse2 = (m_used == -INFINITY) ? -INFINITY : m_used * p.sl2 + log2f(l_sum);
+                p.lse[(size_t)h * p.T + seq_start + i] = lse2 * 0.6931471805599453f;
             }
 #ifdef SWAA_PHASE_TIMING
             if (lane == 0 && wq == 0) {
@@ -690,6 +733,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
 #endif
         }
+        if (lane == 0) tma_store_wait_all();  // outstanding output stores of this warp
     }
 
     // ---- teardown: every thread arrives here (also after a failed wait); free the tensor memory
