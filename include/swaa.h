@@ -87,8 +87,10 @@ int swaa_prefill(const void* q, const void* k, const void* v, void* out, const i
  *   workspace       device scratch of at least swaa_decode_workspace_size(...) bytes for the same
  *                   shape arguments, 256-byte aligned; contents need not be initialised and are
  *                   overwritten.  Two calls that overlap on the GPU must not share a workspace.
- * The visible cache entries are split over thread blocks (split-K); partial results are merged by a
- * log-sum-exp combine inside the same launch.
+ * The visible cache entries of all sequences and heads form one list of 64-entry tiles that is cut
+ * evenly over a persistent grid (split-K across blocks wherever a cut falls inside a sequence);
+ * partial results are merged by a log-sum-exp combine inside the same launch.  Cache entries past
+ * seqlens[b] are never used, whatever they hold.
  */
 size_t swaa_decode_workspace_size(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full);
 
@@ -107,10 +109,11 @@ int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out
  * memory pool, and must not take memory behind its back; a process whose device memory is already
  * handed out in full to other owners.
  *
- *   - The scratch array is SWAA_DECODE_STATIC_SCRATCH_BYTES (16 MiB) per GPU, held by every GPU that
+ *   - The scratch array is SWAA_DECODE_STATIC_SCRATCH_BYTES (2 MiB) per GPU, held by every GPU that
  *     loads the library until the process exits.  A shape whose scratch need
  *     (swaa_decode_workspace_size) exceeds it is rejected with SWAA_ERR_WORKSPACE and nothing runs;
- *     use swaa_decode with a caller-owned workspace for those.
+ *     use swaa_decode with a caller-owned workspace for those (on a 148-SM device: head size 128
+ *     with more than 8 query heads per key/value head, once the batch is large enough to occupy every SM).
  *   - The first call on each device looks up the array's device address (once per device, with that
  *     device current) before it launches.  Make that first call outside any stream capture.
  *   - All calls on one device share the one array, and it keeps whatever the previous call left
@@ -118,7 +121,7 @@ int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out
  *     on the same GPU (different streams, no dependency between them) race on it: serialise them.
  * Returns the same status codes as swaa_decode.
  */
-#define SWAA_DECODE_STATIC_SCRATCH_BYTES (16u << 20)
+#define SWAA_DECODE_STATIC_SCRATCH_BYTES (2u << 20)
 int swaa_decode_static(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
                        int B, int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
                        void* stream);
@@ -160,8 +163,9 @@ int swaa_prefill_tile_needs_mask(int L, int m, int n, int BM, int BN, int window
 int swaa_prefill_block_m(void);
 int swaa_prefill_block_n(void);
 
-/* Number of key splits swaa_decode uses for these arguments on the current device (>= 1). */
-int swaa_decode_num_splits(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full);
+/* Number of thread blocks swaa_decode cuts the visible cache entries over, for these arguments on the
+ * current device (>= 1). */
+int swaa_decode_num_blocks(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full);
 
 /* Static string for a swaa_status value. */
 const char* swaa_status_str(int status);

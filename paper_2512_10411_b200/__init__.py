@@ -8,7 +8,7 @@ unloadable library raises.
 from .binding import (  # noqa: F401
     SwaaError,
     SwaaPolicy,
-    decode_num_splits,
+    decode_num_blocks,
     decode_workspace_size,
     kernel_launch_count,
     prefill_block_shape,

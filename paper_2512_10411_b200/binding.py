@@ -64,8 +64,8 @@ def load_library():
     lib.swaa_prefill.restype = ci
     lib.swaa_decode_workspace_size.argtypes = [ci] * 8
     lib.swaa_decode_workspace_size.restype = ctypes.c_size_t
-    lib.swaa_decode_num_splits.argtypes = [ci] * 8
-    lib.swaa_decode_num_splits.restype = ci
+    lib.swaa_decode_num_blocks.argtypes = [ci] * 8
+    lib.swaa_decode_num_blocks.restype = ci
     lib.swaa_decode.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
     lib.swaa_decode.restype = ci
     lib.swaa_decode_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp]
@@ -137,8 +137,8 @@ def decode_workspace_size(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) -> int:
                                                          int(bool(is_full))))
 
 
-def decode_num_splits(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) -> int:
-    return int(load_library().swaa_decode_num_splits(B, Hq, Hkv, D, Lmax, int(window), int(n_sink),
+def decode_num_blocks(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) -> int:
+    return int(load_library().swaa_decode_num_blocks(B, Hq, Hkv, D, Lmax, int(window), int(n_sink),
                                                      int(bool(is_full))))
 
 
@@ -161,7 +161,7 @@ def swaa_decode(q, kcache, vcache, out, seqlens, window: int, n_sink: int, is_fu
         raise SwaaError(rc, "swaa_decode")
 
 
-DECODE_STATIC_SCRATCH_BYTES = 16 << 20
+DECODE_STATIC_SCRATCH_BYTES = 2 << 20
 
 
 def swaa_decode_static(q, kcache, vcache, out, seqlens, window: int, n_sink: int, is_full: bool, scale: float = 0.0,

@@ -1,51 +1,122 @@
-// Split-K decode attention (one query token per sequence) -- HBM-bound.
+// Decode attention (one query token per sequence) -- HBM-bound streaming kernel.
 //
 // Sec. 3.1.1 ("FA Decode"): the generated token attends to every earlier token, so the kernel
 // streams the whole KV cache of its sequence; an SWA decode step reads the first n_sink entries plus
 // the last `window` entries only.  App. A: the full-context cache is retained for decoding.
 //
-// Work decomposition: one thread block per (key/value head, key split, sequence).  All G = Hq/Hkv
-// query heads of the group are processed together so every K/V byte is read from HBM exactly once.
-// The visible cache entries form one virtual index space [0, n_vis) = sinks ++ window, cut into blocks
-// of 16 keys; a split owns a contiguous run of blocks and its four warps take them round-robin.
+// Work decomposition.  An item is one (sequence, key/value head, chunk of up to 8*NH query heads of
+// that head's group); all query heads of a chunk are processed together so each K/V byte is fetched
+// once.  The visible cache entries of an item are cut into tiles of 64 keys (sink tiles, then window
+// tiles starting at the first window key).  All tiles of all items form one list in (sequence, item,
+// tile) order, and block c of a persistent grid (one block per SM) owns the contiguous run
+// [c * tpc, (c+1) * tpc) of it, so every SM streams the same number of bytes whatever the batch
+// shape.  A block therefore holds at most two incomplete items (the first and the last of its run);
+// it writes complete items straight to `out` and incomplete ones as (max, sum, unnormalised O)
+// partials, which the last block to finish an item merges (atomic ticket, same launch).
 //
-// Data path: each lane reads 16-byte pieces of K/V rows straight into registers (a warp covers whole
-// 256-byte rows, so the loads are fully coalesced), and both contractions run on warp-level tensor
-// core MMAs with fp32 accumulation in the transposed form
+// Data path.  One producer thread keeps a ring of shared-memory stages full with TMA tile copies
+// (K and V boxes of [64 keys][64 channels], 128-byte swizzle), so that the bytes in flight per SM do
+// not depend on registers or occupancy.  Four consumer warps each take 16 keys of every tile and run
+// both contractions on warp-level tensor-core MMAs with fp32 accumulation in the transposed form
 //     S^T[16 keys x 8 heads] = K[16 keys x D] * Q^T[D x 8 heads]
 //     O^T[16 ch  x 8 heads] += V^T[16 ch x 16 keys] * P^T[16 keys x 8 heads]
-// so that the small head count sits in the MMA's N = 8 dimension and no accumulator rows are wasted.
-// The contraction index of the first product is a fixed permutation of the channels, chosen so that
-// an A/B fragment register is exactly one 32-bit word of a 16-byte load (a dot product does not care
-// about the order of its terms).  P^T reaches the second product's B fragment through movmatrix.
-// Partial (max, sum, O) triples of the splits are merged by the last block to finish (atomic ticket).
+// so that the small head count sits in the MMA's N = 8 dimension.  K fragments come from ldmatrix, V^T
+// fragments from ldmatrix.trans, and P^T reaches the second product's B fragment through movmatrix.
+//
+// Every mbarrier wait is bounded; a wait that runs out records SWAA_ERR_TIMEOUT, the consumers finish
+// their loops without computing or storing, and the producer waits (bounded) for its copies in flight.
 #pragma once
 
 #include "swaa_internal.cuh"
+#include "swaa_ptx.cuh"
 
 namespace swaa {
 
 struct DecodeParams {
     const __nv_bfloat16* q;
-    const __nv_bfloat16* kc;
-    const __nv_bfloat16* vc;
     __nv_bfloat16* out;
     const int32_t* seqlens;
     int B, Lmax, Hq, Hkv, G;
     int HG;        // head chunks per kv head (each chunk holds up to 8*NH query heads)
+    int IPB;       // items per sequence = Hkv * HG
     int window, n_sink, is_full;
     float sl2;     // softmax scale * log2(e)
-    int nsplit;
-    int* counters;     // [B * Hkv * HG] tickets, zeroed before the launch
-    float* part_ml;    // [B, Hq, nsplit, 2]  (running max in score units, sum)
-    float* part_o;     // [B, Hq, nsplit, D]  unnormalised
+    int* tickets;  // [gridDim.x], zeroed before the launch
+    float* part;   // [2 * gridDim.x][8*NH][D + 2]: per head (max in score units, sum, unnormalised O)
 };
 
-constexpr int kDecodeWarps = 4;
-constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kDecodeBlockKeys = 16;
+constexpr int kDecodeTileKeys = 64;
+constexpr int kDecodeConsumerWarps = 4;
+constexpr int kDecodeConsumerThreads = kDecodeConsumerWarps * 32;
+constexpr int kDecodeThreads = kDecodeConsumerThreads + 32;  // + the producer warp
+constexpr int kDecodeMinTilesPerBlock = 4;                   // do not cut the list finer than 256 keys
 
-__device__ __forceinline__ uint4 ld_stream16(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
+template <int D, int NH>
+struct DecodeSmem {
+    static constexpr int kPanels = D / 64;
+    static constexpr int kPanelBytes = kDecodeTileKeys * 128;       // [64 keys][64 ch] bf16
+    static constexpr int kTileBytes = kPanels * kPanelBytes;        // one K or V tile
+    static constexpr int kStageBytes = 2 * kTileBytes;              // K then V
+    static constexpr int kHC = 8 * NH;
+    static constexpr int kMergeBytes = kDecodeConsumerWarps * kHC * (D + 1 + 2) * 4;  // O, max, sum per warp
+    static constexpr int kStages = (220 * 1024 - kMergeBytes) / kStageBytes < 12 ? (220 * 1024 - kMergeBytes) / kStageBytes : 12;
+    static constexpr int kOffMerge = kStages * kStageBytes;
+    static constexpr int kOffBar = kOffMerge + ((kMergeBytes + 15) / 16) * 16;
+    static constexpr int kOffMisc = kOffBar + 3 * kStages * 8;
+    static constexpr int kBytes = kOffMisc + 64;
+    static constexpr int kDynamicBytes = kBytes + 1024;  // room to align the base to 1024 B
+};
+
+// Visible part of one sequence's cache, in tiles.
+struct SeqGeom {
+    int len;  // valid entries (0 when seqlens[b] is out of range)
+    int lo;   // first window key
+    int ns;   // sink keys that lie before the window
+    int nst;  // sink tiles
+    int nt;   // tiles per item
+};
+
+__host__ __device__ inline SeqGeom decode_seq_geom(int len, int Lmax, int window, int n_sink, int is_full) {
+    SeqGeom s;
+    if (len < 1 || len > Lmax) {
+        s.len = s.lo = s.ns = s.nst = s.nt = 0;
+        return s;
+    }
+    s.len = len;
+    s.lo = is_full ? 0 : (len > window ? len - window : 0);
+    s.ns = is_full ? 0 : (n_sink < s.lo ? n_sink : s.lo);
+    s.nst = (s.ns + kDecodeTileKeys - 1) / kDecodeTileKeys;
+    s.nt = s.nst + (len - s.lo + kDecodeTileKeys - 1) / kDecodeTileKeys;
+    return s;
+}
+
+// Position in the global tile list; every role of a block walks the same positions.
+struct DecodeWalker {
+    int b, hv, ti;
+    SeqGeom s;
+    __device__ __forceinline__ void seek(const DecodeParams& p, int b0, long long off) {
+        b = b0;
+        s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
+        hv = (int)(off / s.nt);
+        ti = (int)(off - (long long)hv * s.nt);
+    }
+    __device__ __forceinline__ void next(const DecodeParams& p) {
+        if (++ti < s.nt) return;
+        ti = 0;
+        if (++hv < p.IPB) return;
+        hv = 0;
+        while (++b < p.B) {
+            s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
+            if (s.nt > 0) return;
+        }
+        s.nt = 0;  // past the last sequence
+    }
+    __device__ __forceinline__ int key0() const { return ti < s.nst ? ti * kDecodeTileKeys : s.lo + (ti - s.nst) * kDecodeTileKeys; }
+    __device__ __forceinline__ int valid() const {  // visible keys in this tile, 1 .. 64
+        const int left = ti < s.nst ? s.ns - ti * kDecodeTileKeys : s.len - key0();
+        return left < kDecodeTileKeys ? left : kDecodeTileKeys;
+    }
+};
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -61,270 +132,363 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     return d;
 }
 
-__device__ __forceinline__ uint32_t u4_word(const uint4& v, int i) {
-    return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
-}
-
-// 16-bit element e (0..7) of two 16-byte pieces packed as (lo = a[e], hi = b[e]).
-__device__ __forceinline__ uint32_t pair_elem(const uint4& a, const uint4& b, int e) {
-    const uint32_t wa = u4_word(a, e >> 1), wb = u4_word(b, e >> 1);
-    return (e & 1) ? __byte_perm(wa, wb, 0x7632) : __byte_perm(wa, wb, 0x5410);
+__device__ __forceinline__ void consumer_sync() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumerThreads) : "memory");
 }
 
 template <int D, int NH>
-__global__ void __launch_bounds__(kDecodeThreads, 2) decode_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(kDecodeThreads, 1)
+decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const DecodeParams p) {
     static_assert(D == 64 || D == 128, "head size");
-    constexpr int NKI = D / 32;   // 16-byte pieces of one K row per lane
-    constexpr int NCH = D / 64;   // 16-byte pieces of one V row per lane
-    constexpr int NQ = D / 16;    // 16-channel M-blocks of O^T
-    constexpr int HC = 8 * NH;    // query heads per chunk
+    using L = DecodeSmem<D, NH>;
+    constexpr int ST = L::kStages;
+    constexpr int NKK = D / 16;  // 16-channel steps of the first product = 16-channel row blocks of O^T
+    constexpr int HC = L::kHC;   // query heads per chunk
 
-    const int hv = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
-    const int hk = hv / p.HG, ch = hv - hk * p.HG;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
-    const int h0 = hk * p.G + ch * HC;                 // first query head of this chunk
-    const int gc = min(HC, p.G - ch * HC);             // heads in this chunk
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    float* sm_o = reinterpret_cast<float*>(smem_gen + L::kOffMerge);   // [warps][HC][D + 1]
+    float* sm_m = sm_o + kDecodeConsumerWarps * HC * (D + 1);          // [warps][HC]
+    float* sm_l = sm_m + kDecodeConsumerWarps * HC;                    // [warps][HC]
+    const uint32_t bars = smem_base + L::kOffBar;
+    auto bar_kf = [&](int s) -> uint32_t { return bars + 8u * (uint32_t)s; };
+    auto bar_vf = [&](int s) -> uint32_t { return bars + 8u * (uint32_t)(ST + s); };
+    auto bar_e = [&](int s) -> uint32_t { return bars + 8u * (uint32_t)(2 * ST + s); };
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + L::kOffMisc);
+    volatile int* sm_last = abort_flag + 1;
 
-    int len = p.seqlens[b];
-    if (len < 1 || len > p.Lmax) {
-        if (tid == 0) record_device_error(SWAA_ERR_BAD_SEQLENS);
-        len = 0;
-    }
-    const int lo = p.is_full ? 0 : max(0, len - p.window);
-    const int ns = p.is_full ? 0 : min(p.n_sink, lo);
-    const int n_vis = ns + (len - lo);
-    const int nblk = (n_vis + kDecodeBlockKeys - 1) / kDecodeBlockKeys;
-    const int bps = (nblk + p.nsplit - 1) / p.nsplit;
-    const int blk_begin = split * bps;
-    const int blk_end = min(nblk, blk_begin + bps);
+    __shared__ long long sc_scan[kDecodeThreads];
+    __shared__ long long sc_off;
+    __shared__ int sc_b0;
 
-    const size_t row_stride = (size_t)p.Hkv * D;  // elements between consecutive cache entries
-    const __nv_bfloat16* kbase = p.kc + ((size_t)b * p.Lmax * p.Hkv + hk) * D;
-    const __nv_bfloat16* vbase = p.vc + ((size_t)b * p.Lmax * p.Hkv + hk) * D;
-    auto key_of = [&](int v) -> size_t {  // virtual index -> cache entry (clamped to stay in bounds)
-        v = min(v, n_vis - 1);
-        return (size_t)(v < ns ? v : lo + (v - ns));
-    };
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ncta = (int)gridDim.x, cta = (int)blockIdx.x;
 
-    // Q^T fragments: lane (g, c) holds, for head g of each 8-head block, pieces 4i+c of the row.
-    uint4 qf[NH][NKI];
-#pragma unroll
-    for (int nh = 0; nh < NH; ++nh) {
-        const int hh = nh * 8 + g;
-#pragma unroll
-        for (int i = 0; i < NKI; ++i) {
-            if (hh < gc)
-                qf[nh][i] = *reinterpret_cast<const uint4*>(p.q + ((size_t)b * p.Hq + h0 + hh) * D + (4 * i + c) * 8);
-            else
-                qf[nh][i] = make_uint4(0, 0, 0, 0);
-        }
-    }
-
-    float m_run[NH][2], l_run[NH][2], oacc[NH][NQ][4];
-#pragma unroll
-    for (int nh = 0; nh < NH; ++nh) {
-        m_run[nh][0] = m_run[nh][1] = -INFINITY;
-        l_run[nh][0] = l_run[nh][1] = 0.f;
-#pragma unroll
-        for (int qb = 0; qb < NQ; ++qb)
-#pragma unroll
-            for (int r = 0; r < 4; ++r) oacc[nh][qb][r] = 0.f;
-    }
-
-    uint4 kcur[2][NKI], vcur[4][NCH], knext[2][NKI], vnext[4][NCH];
-    auto load_k = [&](int blk, uint4 (&kr)[2][NKI]) {
-        const int v0 = blk * kDecodeBlockKeys;
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const __nv_bfloat16* row = kbase + key_of(v0 + g + 8 * r) * row_stride;
-#pragma unroll
-            for (int i = 0; i < NKI; ++i) kr[r][i] = ld_stream16(row + (4 * i + c) * 8);
-        }
-    };
-    auto load_v = [&](int blk, uint4 (&vr)[4][NCH]) {
-        const int v0 = blk * kDecodeBlockKeys;
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int slot = 2 * c + (r & 1) + 8 * (r >> 1);  // keys 2c, 2c+1, 2c+8, 2c+9
-            const __nv_bfloat16* row = vbase + key_of(v0 + slot) * row_stride;
-#pragma unroll
-            for (int j = 0; j < NCH; ++j) vr[r][j] = ld_stream16(row + (g + 8 * j) * 8);
-        }
-    };
-
-    int blk = blk_begin + warp;
-    if (blk < blk_end) {
-        load_k(blk, kcur);
-        load_v(blk, vcur);
-    }
-    for (; blk < blk_end; blk += kDecodeWarps) {
-        const int nxt = blk + kDecodeWarps;
-        const bool has_next = nxt < blk_end;
-        if (has_next) load_k(nxt, knext);
-
-        // ---- S^T = K Q^T : rows = keys (g, g+8), cols = heads (2c, 2c+1)
-        float sacc[NH][4];
-#pragma unroll
-        for (int nh = 0; nh < NH; ++nh) {
-            sacc[nh][0] = sacc[nh][1] = sacc[nh][2] = sacc[nh][3] = 0.f;
-#pragma unroll
-            for (int i = 0; i < NKI; ++i) {
-                mma_bf16_16816(sacc[nh], kcur[0][i].x, kcur[1][i].x, kcur[0][i].y, kcur[1][i].y, qf[nh][i].x,
-                               qf[nh][i].y);
-                mma_bf16_16816(sacc[nh], kcur[0][i].z, kcur[1][i].z, kcur[0][i].w, kcur[1][i].w, qf[nh][i].z,
-                               qf[nh][i].w);
+    // ---- where does this block's run of the global tile list start?  (scan of tiles per sequence)
+    const int chunk = (p.B + kDecodeThreads - 1) / kDecodeThreads;
+    const int bb = min(p.B, tid * chunk), be = min(p.B, bb + chunk);
+    long long mine = 0;
+    for (int b = bb; b < be; ++b) {
+        const SeqGeom g = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
+        if (g.nt == 0) {
+            record_device_error(SWAA_ERR_BAD_SEQLENS);
+            if (b % ncta == cta) {  // this sequence has no tiles: its output rows are zero-filled here
+                uint4* o = reinterpret_cast<uint4*>(p.out + (size_t)b * p.Hq * D);
+                for (int i = 0; i < p.Hq * D / 8; ++i) o[i] = make_uint4(0, 0, 0, 0);
             }
         }
-        if (has_next) load_v(nxt, vnext);
-
-        // ---- online softmax over the 16 keys of this block
-        const int v0 = blk * kDecodeBlockKeys;
-        const bool ok0 = v0 + g < n_vis, ok1 = v0 + g + 8 < n_vis;
-        uint32_t pb[NH][2];
-#pragma unroll
-        for (int nh = 0; nh < NH; ++nh) {
-            float alpha[2];
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const float s0 = ok0 ? sacc[nh][e] : -INFINITY;
-                const float s1 = ok1 ? sacc[nh][2 + e] : -INFINITY;
-                float bm = fmaxf(s0, s1);
-                bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
-                bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
-                bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
-                const float m_new = fmaxf(m_run[nh][e], bm);  // finite: key v0 is always valid
-                alpha[e] = ex2f((m_run[nh][e] - m_new) * p.sl2);
-                m_run[nh][e] = m_new;
-                const float off = m_new * p.sl2;
-                const float p0 = ex2f(fmaf(s0, p.sl2, -off));
-                const float p1 = ex2f(fmaf(s1, p.sl2, -off));
-                l_run[nh][e] = l_run[nh][e] * alpha[e] + p0 + p1;
-                sacc[nh][e] = p0;
-                sacc[nh][2 + e] = p1;
+        mine += (long long)g.nt * p.IPB;
+    }
+    sc_scan[tid] = mine;
+    __syncthreads();
+    for (int off = 1; off < kDecodeThreads; off <<= 1) {
+        const long long v = tid >= off ? sc_scan[tid - off] : 0;
+        __syncthreads();
+        sc_scan[tid] += v;
+        __syncthreads();
+    }
+    const long long total = sc_scan[kDecodeThreads - 1];
+    long long tpc = (total + ncta - 1) / ncta;
+    if (tpc < kDecodeMinTilesPerBlock) tpc = kDecodeMinTilesPerBlock;
+    const long long t0 = (long long)cta * tpc;
+    const long long t1 = total < t0 + tpc ? total : t0 + tpc;
+    if (t0 >= t1) return;  // nothing for this block (uniform: no barrier is pending)
+    if (sc_scan[tid] - mine <= t0 && t0 < sc_scan[tid]) {
+        long long acc = sc_scan[tid] - mine;
+        for (int b = bb; b < be; ++b) {
+            const SeqGeom g = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
+            const long long nb = (long long)g.nt * p.IPB;
+            if (t0 < acc + nb) {
+                sc_b0 = b;
+                sc_off = t0 - acc;
+                break;
             }
-            if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+            acc += nb;
+        }
+    }
+    if (tid == 0) {
+        *abort_flag = 0;
+        *sm_last = 0;
+        for (int s = 0; s < ST; ++s) {
+            mbar_init(bar_kf(s), 1u);
+            mbar_init(bar_vf(s), 1u);
+            mbar_init(bar_e(s), (uint32_t)kDecodeConsumerWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int cnt = (int)(t1 - t0);  // tpc <= tiles of the whole problem / blocks, far below 2^31 in practice
+    const int b0 = sc_b0;
+    const long long off0 = sc_off;
+
+    if (warp == kDecodeConsumerWarps) {
+        // =========================================================================== TMA producer
+        if (lane == 0) {
+            DecodeWalker w;
+            w.seek(p, b0, off0);
+            bool ok = true;
+            int n = 0, s = 0;
+            uint32_t ph = 0;
+            for (; n < cnt; ++n, w.next(p)) {
+                ok = mbar_wait(bar_e(s), ph ^ 1u, abort_flag);
+                if (!ok) break;
+                const int key0 = w.key0(), hk = w.hv / p.HG;
+                const uint32_t dst = smem_base + (uint32_t)s * L::kStageBytes;
+                mbar_arrive_expect_tx(bar_kf(s), (uint32_t)L::kTileBytes);
 #pragma unroll
-                for (int qb = 0; qb < NQ; ++qb) {
-                    oacc[nh][qb][0] *= alpha[0];
-                    oacc[nh][qb][1] *= alpha[1];
-                    oacc[nh][qb][2] *= alpha[0];
-                    oacc[nh][qb][3] *= alpha[1];
+                for (int pn = 0; pn < L::kPanels; ++pn)
+                    tma_load_4d(dst + pn * L::kPanelBytes, &tm_k, pn * 64, hk, key0, w.b, bar_kf(s));
+                mbar_arrive_expect_tx(bar_vf(s), (uint32_t)L::kTileBytes);
+#pragma unroll
+                for (int pn = 0; pn < L::kPanels; ++pn)
+                    tma_load_4d(dst + L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, key0, w.b, bar_vf(s));
+                if (++s == ST) {
+                    s = 0;
+                    ph ^= 1u;
                 }
             }
-            // P^T as the B fragment: (keys 2c, 2c+1 | 2c+8, 2c+9 ; head g)
-            pb[nh][0] = movmatrix_trans(pack_bf16x2(sacc[nh][0], sacc[nh][1]));
-            pb[nh][1] = movmatrix_trans(pack_bf16x2(sacc[nh][2], sacc[nh][3]));
-        }
-
-        // ---- O^T += V^T P^T : rows = channels, cols = heads
-#pragma unroll
-        for (int qb = 0; qb < NQ; ++qb) {
-            uint32_t a0, a1, a2, a3;
-            if (D == 128) {  // rows g -> channel 8g+qb (piece g), rows g+8 -> channel 8(g+8)+qb (piece g+8)
-                a0 = pair_elem(vcur[0][0], vcur[1][0], qb);
-                a1 = pair_elem(vcur[0][NCH - 1], vcur[1][NCH - 1], qb);
-                a2 = pair_elem(vcur[2][0], vcur[3][0], qb);
-                a3 = pair_elem(vcur[2][NCH - 1], vcur[3][NCH - 1], qb);
-            } else {         // one piece per row: rows g -> channel 8g+qb, rows g+8 -> channel 8g+4+qb
-                a0 = pair_elem(vcur[0][0], vcur[1][0], qb);
-                a1 = pair_elem(vcur[0][0], vcur[1][0], qb + 4);
-                a2 = pair_elem(vcur[2][0], vcur[3][0], qb);
-                a3 = pair_elem(vcur[2][0], vcur[3][0], qb + 4);
-            }
-#pragma unroll
-            for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(oacc[nh][qb], a0, a1, a2, a3, pb[nh][0], pb[nh][1]);
-        }
-
-        if (has_next) {
-#pragma unroll
-            for (int r = 0; r < 2; ++r)
-#pragma unroll
-                for (int i = 0; i < NKI; ++i) kcur[r][i] = knext[r][i];
-#pragma unroll
-            for (int r = 0; r < 4; ++r)
-#pragma unroll
-                for (int j = 0; j < NCH; ++j) vcur[r][j] = vnext[r][j];
-        }
-    }
-
-    // ---- merge the four warps of the block through shared memory
-    __shared__ float sm_m[kDecodeWarps][HC], sm_l[kDecodeWarps][HC];
-    __shared__ float sm_o[kDecodeWarps][HC][D + 1];
-    __shared__ int sm_last;
-#pragma unroll
-    for (int nh = 0; nh < NH; ++nh) {
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            float l = l_run[nh][e];
-            l += __shfl_xor_sync(0xffffffffu, l, 4);
-            l += __shfl_xor_sync(0xffffffffu, l, 8);
-            l += __shfl_xor_sync(0xffffffffu, l, 16);
-            const int hh = nh * 8 + 2 * c + e;
-            if (g == 0) {
-                sm_m[warp][hh] = m_run[nh][e];
-                sm_l[warp][hh] = l;
-            }
-#pragma unroll
-            for (int qb = 0; qb < NQ; ++qb) {
-                const int dA = (D == 128) ? 8 * g + qb : 8 * g + qb;
-                const int dB = (D == 128) ? 8 * (g + 8) + qb : 8 * g + 4 + qb;
-                sm_o[warp][hh][dA] = oacc[nh][qb][e];
-                sm_o[warp][hh][dB] = oacc[nh][qb][2 + e];
+            if (!ok) {
+                // give the copies in flight a bounded chance to land before the block's memory is released
+                const uint64_t tw = global_timer_ns();
+                bool landed = false;
+                while (!landed && global_timer_ns() - tw < kWaitLimitNs) {
+                    landed = true;
+                    for (int m = max(0, n - ST); m < n; ++m) {
+                        landed = landed && mbar_try_wait(bar_kf(m % ST), (uint32_t)(m / ST) & 1u);
+                        landed = landed && mbar_try_wait(bar_vf(m % ST), (uint32_t)(m / ST) & 1u);
+                    }
+                }
             }
         }
+        return;
     }
-    __syncthreads();
 
-    const bool direct = p.nsplit == 1;
-    for (int idx = tid; idx < gc * D; idx += kDecodeThreads) {
-        const int hh = idx / D, d = idx - hh * D;
-        float M = -INFINITY;
+    // ============================================================================== consumers
+    const int g = lane >> 2, c = lane & 3;
+    // ldmatrix row addresses inside a tile (byte offset of the row, and the row's swizzle key)
+    const int krow = 16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1);  // K: matrices (keys lo/hi) x (channels lo/hi)
+    const int kchk = lane >> 4;
+    const int vrow = 16 * warp + (lane & 7) + 8 * (lane >> 4);        // V: matrices (channels lo/hi) x (keys lo/hi)
+    const int vchk = (lane >> 3) & 1;
+
+    DecodeWalker w;
+    w.seek(p, b0, off0);
+    bool ok = true;
+    bool first_seg = true;
+    int n = 0, s = 0;
+    uint32_t ph = 0;
+    while (n < cnt) {
+        // ---- one segment: the tiles of the current item that belong to this block
+        const int b = w.b, hv = w.hv, ti_begin = w.ti, nt = w.s.nt;
+        const int seg_tiles = min(cnt - n, nt - ti_begin);
+        const long long seg_t0 = t0 + n;
+        const int hk = hv / p.HG, ch = hv - hk * p.HG;
+        const int h0 = hk * p.G + ch * HC;      // first query head of this chunk
+        const int gc = min(HC, p.G - ch * HC);  // heads in this chunk
+
+        // Q^T fragments (B operand): lane (g, c) holds channels 16kk + 2c, +1 and 16kk + 2c + 8, +9 of head g
+        uint32_t qf[NH][NKK][2];
 #pragma unroll
-        for (int w = 0; w < kDecodeWarps; ++w) M = fmaxf(M, sm_m[w][hh]);
-        float den = 0.f, num = 0.f;
+        for (int nh = 0; nh < NH; ++nh) {
+            const int hh = nh * 8 + g;
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((size_t)b * p.Hq + h0 + (hh < gc ? hh : 0)) * D);
 #pragma unroll
-        for (int w = 0; w < kDecodeWarps; ++w) {
-            const float wgt = sm_m[w][hh] == -INFINITY ? 0.f : ex2f((sm_m[w][hh] - M) * p.sl2);
-            den += wgt * sm_l[w][hh];
-            num += wgt * sm_o[w][hh][d];
-        }
-        const size_t row = (size_t)b * p.Hq + h0 + hh;
-        if (direct) {
-            p.out[row * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
-        } else {
-            p.part_o[(row * p.nsplit + split) * D + d] = num;
-            if (d == 0) {
-                p.part_ml[(row * p.nsplit + split) * 2 + 0] = M;
-                p.part_ml[(row * p.nsplit + split) * 2 + 1] = den;
+            for (int kk = 0; kk < NKK; ++kk) {
+                qf[nh][kk][0] = hh < gc ? __ldg(qrow + kk * 8 + c) : 0u;
+                qf[nh][kk][1] = hh < gc ? __ldg(qrow + kk * 8 + c + 4) : 0u;
             }
         }
-    }
-    if (direct) return;
-
-    // ---- the last block of this (sequence, head chunk) to arrive merges the splits
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int ticket = atomicAdd(&p.counters[b * gridDim.x + hv], 1);
-        sm_last = (ticket == p.nsplit - 1);
-    }
-    __syncthreads();
-    if (!sm_last) return;
-    __threadfence();
-    for (int idx = tid; idx < gc * D; idx += kDecodeThreads) {
-        const int hh = idx / D, d = idx - hh * D;
-        const size_t row = (size_t)b * p.Hq + h0 + hh;
-        const float* ml = p.part_ml + row * p.nsplit * 2;
-        float M = -INFINITY;
-        for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, __ldcg(ml + 2 * s));
-        float den = 0.f, num = 0.f;
-        for (int s = 0; s < p.nsplit; ++s) {
-            const float ms = __ldcg(ml + 2 * s);
-            const float wgt = ms == -INFINITY ? 0.f : ex2f((ms - M) * p.sl2);
-            den += wgt * __ldcg(ml + 2 * s + 1);
-            num += wgt * __ldcg(p.part_o + (row * p.nsplit + s) * D + d);
+        float m_run[NH][2], l_run[NH][2], oacc[NH][NKK][4];
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh) {
+            m_run[nh][0] = m_run[nh][1] = -INFINITY;
+            l_run[nh][0] = l_run[nh][1] = 0.f;
+#pragma unroll
+            for (int qb = 0; qb < NKK; ++qb)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) oacc[nh][qb][r] = 0.f;
         }
-        p.out[row * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+
+        for (int j = 0; j < seg_tiles; ++j, ++n, w.next(p)) {
+            const int vw = w.valid() - 16 * warp;  // visible keys among this warp's 16
+            const uint32_t stage = smem_base + (uint32_t)s * L::kStageBytes;
+            ok = ok && mbar_wait(bar_kf(s), ph, abort_flag);
+            if (ok && vw > 0) {
+                // ---- S^T = K Q^T : rows = keys (g, g+8), cols = heads (2c, 2c+1)
+                float sacc[NH][4];
+#pragma unroll
+                for (int nh = 0; nh < NH; ++nh) sacc[nh][0] = sacc[nh][1] = sacc[nh][2] = sacc[nh][3] = 0.f;
+#pragma unroll
+                for (int kk = 0; kk < NKK; ++kk) {
+                    const int chunk16 = 2 * kk + kchk;
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4(stage + (uint32_t)((chunk16 >> 3) * L::kPanelBytes + krow * 128 +
+                                                   (((chunk16 & 7) ^ (krow & 7)) << 4)),
+                                a0, a1, a2, a3);
+#pragma unroll
+                    for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(sacc[nh], a0, a1, a2, a3, qf[nh][kk][0], qf[nh][kk][1]);
+                }
+
+                // ---- online softmax over this warp's 16 keys
+                const bool ok0 = g < vw, ok1 = g + 8 < vw;
+                uint32_t pb[NH][2];
+#pragma unroll
+                for (int nh = 0; nh < NH; ++nh) {
+                    float alpha[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float s0 = ok0 ? sacc[nh][e] : -INFINITY;
+                        const float s1 = ok1 ? sacc[nh][2 + e] : -INFINITY;
+                        float bm = fmaxf(s0, s1);
+                        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
+                        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+                        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
+                        const float m_new = fmaxf(m_run[nh][e], bm);  // finite: the warp's first key is visible
+                        alpha[e] = ex2f((m_run[nh][e] - m_new) * p.sl2);
+                        m_run[nh][e] = m_new;
+                        const float off = m_new * p.sl2;
+                        const float p0 = ex2f(fmaf(s0, p.sl2, -off));
+                        const float p1 = ex2f(fmaf(s1, p.sl2, -off));
+                        l_run[nh][e] = l_run[nh][e] * alpha[e] + p0 + p1;
+                        sacc[nh][e] = p0;
+                        sacc[nh][2 + e] = p1;
+                    }
+                    if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+#pragma unroll
+                        for (int qb = 0; qb < NKK; ++qb) {
+                            oacc[nh][qb][0] *= alpha[0];
+                            oacc[nh][qb][1] *= alpha[1];
+                            oacc[nh][qb][2] *= alpha[0];
+                            oacc[nh][qb][3] *= alpha[1];
+                        }
+                    }
+                    // P^T as the B fragment: (keys 2c, 2c+1 | 2c+8, 2c+9 ; head g)
+                    pb[nh][0] = movmatrix_trans(pack_bf16x2(sacc[nh][0], sacc[nh][1]));
+                    pb[nh][1] = movmatrix_trans(pack_bf16x2(sacc[nh][2], sacc[nh][3]));
+                }
+
+                // ---- O^T += V^T P^T : rows = channels (16qb + g, 16qb + g + 8), cols = heads (2c, 2c+1)
+                ok = mbar_wait(bar_vf(s), ph, abort_flag);
+                if (ok) {
+                    // rows of the tile past the last visible key may hold anything (also NaN): clear them
+                    const uint32_t mlo = (2 * c < vw ? 0x0000ffffu : 0u) | (2 * c + 1 < vw ? 0xffff0000u : 0u);
+                    const uint32_t mhi = (2 * c + 8 < vw ? 0x0000ffffu : 0u) | (2 * c + 9 < vw ? 0xffff0000u : 0u);
+#pragma unroll
+                    for (int qb = 0; qb < NKK; ++qb) {
+                        const int chunk16 = 2 * qb + vchk;
+                        uint32_t a0, a1, a2, a3;
+                        ldmatrix_x4_trans(stage + (uint32_t)(L::kTileBytes + (chunk16 >> 3) * L::kPanelBytes + vrow * 128 +
+                                                             (((chunk16 & 7) ^ (vrow & 7)) << 4)),
+                                          a0, a1, a2, a3);
+                        if (vw < 16) {
+                            a0 &= mlo;
+                            a1 &= mlo;
+                            a2 &= mhi;
+                            a3 &= mhi;
+                        }
+#pragma unroll
+                        for (int nh = 0; nh < NH; ++nh) mma_bf16_16816(oacc[nh][qb], a0, a1, a2, a3, pb[nh][0], pb[nh][1]);
+                    }
+                }
+            } else {
+                ok = ok && mbar_wait(bar_vf(s), ph, abort_flag);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_e(s));
+            if (++s == ST) {
+                s = 0;
+                ph ^= 1u;
+            }
+        }
+
+        // ---- merge the four warps of the block through shared memory
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                float l = l_run[nh][e];
+                l += __shfl_xor_sync(0xffffffffu, l, 4);
+                l += __shfl_xor_sync(0xffffffffu, l, 8);
+                l += __shfl_xor_sync(0xffffffffu, l, 16);
+                const int hh = nh * 8 + 2 * c + e;
+                if (g == 0) {
+                    sm_m[warp * HC + hh] = m_run[nh][e];
+                    sm_l[warp * HC + hh] = l;
+                }
+                float* orow = sm_o + (size_t)(warp * HC + hh) * (D + 1);
+#pragma unroll
+                for (int qb = 0; qb < NKK; ++qb) {
+                    orow[16 * qb + g] = oacc[nh][qb][e];
+                    orow[16 * qb + g + 8] = oacc[nh][qb][2 + e];
+                }
+            }
+        }
+        consumer_sync();
+
+        const bool complete = ti_begin == 0 && seg_tiles == nt;
+        const int slot = 2 * cta + (first_seg ? 0 : 1);
+        float* my_part = p.part + (size_t)slot * HC * (D + 2);
+        for (int idx = tid; idx < gc * D; idx += kDecodeConsumerThreads) {
+            const int hh = idx / D, d = idx - hh * D;
+            float M = -INFINITY;
+#pragma unroll
+            for (int wi = 0; wi < kDecodeConsumerWarps; ++wi) M = fmaxf(M, sm_m[wi * HC + hh]);
+            float den = 0.f, num = 0.f;
+#pragma unroll
+            for (int wi = 0; wi < kDecodeConsumerWarps; ++wi) {
+                const float mw = sm_m[wi * HC + hh];
+                const float wgt = mw == -INFINITY ? 0.f : ex2f((mw - M) * p.sl2);
+                den += wgt * sm_l[wi * HC + hh];
+                num += wgt * sm_o[(size_t)(wi * HC + hh) * (D + 1) + d];
+            }
+            if (!ok) continue;
+            if (complete) {
+                p.out[((size_t)b * p.Hq + h0 + hh) * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+            } else {
+                my_part[hh * (D + 2) + 2 + d] = num;
+                if (d == 0) {
+                    my_part[hh * (D + 2) + 0] = M;
+                    my_part[hh * (D + 2) + 1] = den;
+                }
+            }
+        }
+        if (!complete) {
+            // ---- the last block of this item to arrive merges the item's partials
+            const long long T0 = seg_t0 - ti_begin, T1 = T0 + nt;
+            const int c_first = (int)(T0 / tpc), c_last = (int)((T1 - 1) / tpc);
+            __threadfence();
+            consumer_sync();
+            if (tid == 0) {
+                const int ticket = atomicAdd(&p.tickets[c_first], 1);
+                *sm_last = (ticket == c_last - c_first) ? 1 : 0;
+            }
+            consumer_sync();
+            if (*sm_last && ok) {
+                __threadfence();
+                const bool first_is_slot1 = (long long)c_first * tpc != T0;
+                for (int idx = tid; idx < gc * D; idx += kDecodeConsumerThreads) {
+                    const int hh = idx / D, d = idx - hh * D;
+                    float M = -INFINITY;
+                    for (int cc = c_first; cc <= c_last; ++cc) {
+                        const int sl = 2 * cc + ((cc == c_first && first_is_slot1) ? 1 : 0);
+                        M = fmaxf(M, __ldcg(p.part + ((size_t)sl * HC + hh) * (D + 2)));
+                    }
+                    float den = 0.f, num = 0.f;
+                    for (int cc = c_first; cc <= c_last; ++cc) {
+                        const int sl = 2 * cc + ((cc == c_first && first_is_slot1) ? 1 : 0);
+                        const float* pp = p.part + ((size_t)sl * HC + hh) * (D + 2);
+                        const float ms = __ldcg(pp);
+                        const float wgt = ms == -INFINITY ? 0.f : ex2f((ms - M) * p.sl2);
+                        den += wgt * __ldcg(pp + 1);
+                        num += wgt * __ldcg(pp + 2 + d);
+                    }
+                    p.out[((size_t)b * p.Hq + h0 + hh) * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+                }
+            }
+        }
+        consumer_sync();  // the merge buffers are free for the next segment
+        first_seg = false;
     }
 }
 

@@ -43,14 +43,14 @@ static int current_device_info(DeviceInfo* out) {
 
 // ------------------------------------------------------------------------------------------ decode
 struct DecodePlan {
-    int NH;        // 8-head blocks per chunk (1 or 2)
-    int HG;        // chunks per kv head
-    int nsplit;
-    size_t off_ml, off_o, bytes;
+    int NH;      // 8-head blocks per chunk (1 or 2)
+    int HG;      // chunks per kv head
+    int blocks;  // persistent grid size
+    size_t off_part, bytes;
 };
 
-// Chooses the number of key splits so that the grid fills the machine in whole waves while every
-// block still streams a few hundred keys.  Depends only on the shape arguments and the SM count.
+// One block per SM, fewer when the whole problem has fewer tiles than that.  Depends only on the
+// shape arguments and the SM count (sequence lengths are read on the device).
 static DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full,
                               int sm_count) {
     DecodePlan pl;
@@ -58,37 +58,16 @@ static DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int Lmax, int windo
     pl.NH = G > 8 ? 2 : 1;
     const int HC = 8 * pl.NH;
     pl.HG = (G + HC - 1) / HC;
-    long long n_vis_max = Lmax;
-    if (!is_full) {
-        long long ws = (long long)window + (long long)n_sink;
-        if (ws < n_vis_max) n_vis_max = ws;
-    }
-    const long long nblk = (n_vis_max + kDecodeBlockKeys - 1) / kDecodeBlockKeys;
-    const long long base = (long long)B * Hkv * pl.HG;
-    const long long capacity = (long long)(sm_count > 0 ? sm_count : 148) * 2;  // resident blocks
-    const long long min_blocks_per_split = 4LL * kDecodeWarps;                  // >= 256 keys per block
-    long long max_ns = nblk / min_blocks_per_split;
-    if (max_ns < 1) max_ns = 1;
-    if (max_ns > 64) max_ns = 64;
-    int best = 1;
-    double best_score = -1.0;
-    for (long long ns = 1; ns <= max_ns; ++ns) {
-        const double waves = (double)(base * ns) / (double)capacity;
-        const double eff = waves / ceil(waves);
-        // prefer full waves; among equals prefer more (smaller) blocks up to about four waves
-        const double score = eff + 0.02 * (waves < 4.0 ? waves : 4.0);
-        if (score > best_score + 1e-9) {
-            best_score = score;
-            best = (int)ns;
-        }
-    }
-    pl.nsplit = best;
-    const size_t counters = ((size_t)base * sizeof(int) + 255) / 256 * 256;
-    const size_t ml = (((size_t)B * Hq * pl.nsplit * 2 * sizeof(float)) + 255) / 256 * 256;
-    const size_t o = (size_t)B * Hq * pl.nsplit * D * sizeof(float);
-    pl.off_ml = counters;
-    pl.off_o = counters + ml;
-    pl.bytes = counters + ml + o;
+    const SeqGeom longest = decode_seq_geom(Lmax, Lmax, window, n_sink, is_full);
+    // upper bound on the tiles of one item: a shorter sequence may have one more (ragged) sink tile
+    const long long tiles_ub = (long long)B * Hkv * pl.HG * ((long long)longest.nt + 1);
+    long long blocks = (tiles_ub + kDecodeMinTilesPerBlock - 1) / kDecodeMinTilesPerBlock;
+    const long long sms = sm_count > 0 ? sm_count : 148;
+    if (blocks > sms) blocks = sms;
+    if (blocks < 1) blocks = 1;
+    pl.blocks = (int)blocks;
+    pl.off_part = ((size_t)pl.blocks * sizeof(int) + 255) / 256 * 256;
+    pl.bytes = pl.off_part + (size_t)2 * pl.blocks * HC * (D + 2) * sizeof(float);
     return pl;
 }
 
@@ -96,87 +75,8 @@ static int check_decode_shape(int B, int Hq, int Hkv, int D, int Lmax, int windo
     if (B < 0 || Lmax < 1 || Hq < 1 || Hkv < 1 || n_sink < 0) return SWAA_ERR_INVALID_ARG;
     if (!is_full && window < 1) return SWAA_ERR_INVALID_ARG;
     if (Hq % Hkv != 0 || (D != 64 && D != 128)) return SWAA_ERR_UNSUPPORTED;
-    if (B > 65535) return SWAA_ERR_UNSUPPORTED;  // grid.z limit
     return SWAA_OK;
 }
-
-}  // namespace swaa
-
-using namespace swaa;
-
-extern "C" size_t swaa_decode_workspace_size(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink,
-                                             int is_full) {
-    if (check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) != SWAA_OK || B == 0) return 256;
-    DeviceInfo info;
-    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
-    return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count).bytes;
-}
-
-extern "C" int swaa_decode_num_splits(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink,
-                                      int is_full) {
-    if (check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) != SWAA_OK || B == 0) return 1;
-    DeviceInfo info;
-    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
-    return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count).nsplit;
-}
-
-extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
-                           int B, int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
-                           void* workspace, size_t workspace_bytes, void* stream) {
-    int rc = check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full);
-    if (rc != SWAA_OK) return rc;
-    if (B == 0) return SWAA_OK;
-    if (!q || !kcache || !vcache || !out || !seqlens) return SWAA_ERR_INVALID_ARG;
-    if (!aligned16(q) || !aligned16(kcache) || !aligned16(vcache) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) != 0) return SWAA_ERR_INVALID_ARG;
-    DeviceInfo info;
-    rc = current_device_info(&info);
-    if (rc != SWAA_OK) return rc;
-    if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
-    const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count);
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < pl.bytes)
-        return SWAA_ERR_WORKSPACE;
-
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    DecodeParams p;
-    p.q = static_cast<const __nv_bfloat16*>(q);
-    p.kc = static_cast<const __nv_bfloat16*>(kcache);
-    p.vc = static_cast<const __nv_bfloat16*>(vcache);
-    p.out = static_cast<__nv_bfloat16*>(out);
-    p.seqlens = seqlens;
-    p.B = B;
-    p.Lmax = Lmax;
-    p.Hq = Hq;
-    p.Hkv = Hkv;
-    p.G = Hq / Hkv;
-    p.HG = pl.HG;
-    p.window = window;
-    p.n_sink = n_sink;
-    p.is_full = is_full ? 1 : 0;
-    const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
-    p.sl2 = sc * 1.4426950408889634f;
-    p.nsplit = pl.nsplit;
-    char* ws = static_cast<char*>(workspace);
-    p.counters = reinterpret_cast<int*>(ws);
-    p.part_ml = reinterpret_cast<float*>(ws + pl.off_ml);
-    p.part_o = reinterpret_cast<float*>(ws + pl.off_o);
-    if (pl.nsplit > 1) {
-        if (cudaMemsetAsync(p.counters, 0, pl.off_ml, st) != cudaSuccess) return SWAA_ERR_CUDA;
-    }
-    const dim3 grid((unsigned)(Hkv * pl.HG), (unsigned)pl.nsplit, (unsigned)B);
-    if (D == 128) {
-        if (pl.NH == 1) decode_kernel<128, 1><<<grid, kDecodeThreads, 0, st>>>(p);
-        else decode_kernel<128, 2><<<grid, kDecodeThreads, 0, st>>>(p);
-    } else {
-        if (pl.NH == 1) decode_kernel<64, 1><<<grid, kDecodeThreads, 0, st>>>(p);
-        else decode_kernel<64, 2><<<grid, kDecodeThreads, 0, st>>>(p);
-    }
-    launch_counter().fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
-}
-
-// ----------------------------------------------------------------------------------------- prefill
-namespace swaa {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -197,6 +97,106 @@ static EncodeTiledFn encode_tiled_fn() {
     }
     return fn;
 }
+
+// Tensor map over a bf16 cache [B, Lmax, Hkv, D]: dimensions (D, Hkv, Lmax, B) innermost first; one box
+// is [64 entries] x [1 head] x [64 channels] = 64 rows of 128 bytes, written with the 128-byte swizzle.
+// Rows past Lmax are filled with zeros.
+static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, int Hkv, int D) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return SWAA_ERR_CUDA;
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)Lmax, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)Hkv * D * 2, (cuuint64_t)Lmax * Hkv * D * 2};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)kDecodeTileKeys, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
+template <int D, int NH>
+static int launch_decode(const CUtensorMap& tk, const CUtensorMap& tv, const DecodeParams& p, int blocks,
+                         cudaStream_t st) {
+    using L = DecodeSmem<D, NH>;
+    if (cudaFuncSetAttribute(decode_kernel<D, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
+        cudaSuccess)
+        return SWAA_ERR_CUDA;
+    decode_kernel<D, NH><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tk, tv, p);
+    launch_counter().fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
+}  // namespace swaa
+
+using namespace swaa;
+
+extern "C" size_t swaa_decode_workspace_size(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink,
+                                             int is_full) {
+    if (check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) != SWAA_OK || B == 0) return 256;
+    DeviceInfo info;
+    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
+    return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count).bytes;
+}
+
+extern "C" int swaa_decode_num_blocks(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink,
+                                      int is_full) {
+    if (check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) != SWAA_OK || B == 0) return 1;
+    DeviceInfo info;
+    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
+    return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count).blocks;
+}
+
+extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
+                           int B, int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full);
+    if (rc != SWAA_OK) return rc;
+    if (B == 0) return SWAA_OK;
+    if (!q || !kcache || !vcache || !out || !seqlens) return SWAA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(kcache) || !aligned16(vcache) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) != 0) return SWAA_ERR_INVALID_ARG;
+    DeviceInfo info;
+    rc = current_device_info(&info);
+    if (rc != SWAA_OK) return rc;
+    if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
+    const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < pl.bytes)
+        return SWAA_ERR_WORKSPACE;
+
+    CUtensorMap tk, tv;
+    if ((rc = make_cache_map(&tk, kcache, B, Lmax, Hkv, D)) != SWAA_OK) return rc;
+    if ((rc = make_cache_map(&tv, vcache, B, Lmax, Hkv, D)) != SWAA_OK) return rc;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    DecodeParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.seqlens = seqlens;
+    p.B = B;
+    p.Lmax = Lmax;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = Hq / Hkv;
+    p.HG = pl.HG;
+    p.IPB = Hkv * pl.HG;
+    p.window = window;
+    p.n_sink = n_sink;
+    p.is_full = is_full ? 1 : 0;
+    const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
+    p.sl2 = sc * 1.4426950408889634f;
+    char* ws = static_cast<char*>(workspace);
+    p.tickets = reinterpret_cast<int*>(ws);
+    p.part = reinterpret_cast<float*>(ws + pl.off_part);
+    if (pl.blocks > 1) {
+        if (cudaMemsetAsync(p.tickets, 0, pl.off_part, st) != cudaSuccess) return SWAA_ERR_CUDA;
+    }
+    if (D == 128)
+        return pl.NH == 1 ? launch_decode<128, 1>(tk, tv, p, pl.blocks, st) : launch_decode<128, 2>(tk, tv, p, pl.blocks, st);
+    return pl.NH == 1 ? launch_decode<64, 1>(tk, tv, p, pl.blocks, st) : launch_decode<64, 2>(tk, tv, p, pl.blocks, st);
+}
+
+// ----------------------------------------------------------------------------------------- prefill
+namespace swaa {
 
 // Tensor map over a token-major bf16 tensor [T, H, D]: dimensions (D, H, T) innermost first; one box is
 // [128 tokens] x [1 head] x [64 channels] = 128 rows of 128 bytes, written with the 128-byte swizzle.
@@ -321,8 +321,8 @@ extern "C" int swaa_decode_static(const void* q, const void* kcache, const void*
     void* scratch = nullptr;
     const int rs = decode_static_scratch(&scratch);
     if (rs != SWAA_OK) return rs;
-    // Same kernel and same plan as swaa_decode; its ticket counters (the only part that must start at
-    // zero) are cleared by that call on `stream` before the kernel runs.
+    // Same kernel and same plan as swaa_decode; its tickets (the only part that must start at zero) are
+    // cleared by that call on `stream` before the kernel runs.
     return swaa_decode(q, kcache, vcache, out, seqlens, B, Lmax, Hq, Hkv, D, window, n_sink, is_full, scale, scratch,
                        SWAA_DECODE_STATIC_SCRATCH_BYTES, stream);
 }

@@ -91,6 +91,37 @@ def test_decode_visible_set_is_bit_exact():
             assert np.array_equal(seen[b], want), (W, S, full, b)
 
 
+def test_decode_never_uses_cache_entries_past_seqlens():
+    """Entries past seqlens[b] hold NaN: they share 64-entry tiles with visible entries and must not leak."""
+    cfg = inputs.DecodeConfig("t", 3, 700, 8, 2, 128, 0, 0, seed=21, seqlens=(650, 3, 129))
+    q, kc, vc, seqlens = inputs.make_decode_inputs(cfg, "cuda")
+    for b, n in enumerate(cfg.seqlens):
+        kc[b, n:] = float("nan")
+        vc[b, n:] = float("nan")
+    qh, kh, vh = inputs.to_f32_numpy(q), inputs.to_f32_numpy(kc), inputs.to_f32_numpy(vc)
+    for W, S, full in ((1, 0, True), (100, 4, False), (64, 0, False), (1, 0, False)):
+        out, status = _run_decode(q, kc, vc, seqlens, W, S, full)
+        assert status == 0
+        ref = oracle.decode(qh, kh, vh, cfg.seqlens, W, S, full)
+        check_against_oracle(out, ref["out"], f"NaN tail W={W} S={S} full={full}")
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_decode_many_short_sequences(D):
+    """More sequences than threads in a block, random lengths: many whole items per block, few cut ones."""
+    rng = np.random.default_rng(33)
+    B, Lmax = 437, 260
+    sl = tuple(int(x) for x in rng.integers(1, Lmax + 1, B))
+    cfg = inputs.DecodeConfig("t", B, Lmax, 8, 2, D, 0, 0, seed=34, seqlens=sl)
+    q, kc, vc, seqlens = inputs.make_decode_inputs(cfg, "cuda")
+    qh, kh, vh = inputs.to_f32_numpy(q), inputs.to_f32_numpy(kc), inputs.to_f32_numpy(vc)
+    for W, S, full in ((1, 0, True), (70, 5, False), (128, 100, False)):
+        out, status = _run_decode(q, kc, vc, seqlens, W, S, full)
+        assert status == 0
+        ref = oracle.decode(qh, kh, vh, sl, W, S, full)
+        check_against_oracle(out, ref["out"], f"many sequences D={D} W={W} S={S} full={full}")
+
+
 def test_decode_reports_bad_seqlens_and_zero_fills():
     cfg = inputs.DecodeConfig("t", 3, 128, 4, 2, 64, 0, 0, seed=9, seqlens=(128, 0, 129))
     q, kc, vc, seqlens = inputs.make_decode_inputs(cfg, "cuda")

@@ -115,8 +115,13 @@ def test_status_strings():
 
 
 def test_decode_split_plan_is_consistent():
-    for args in ((16, 32, 8, 128, 65536, 4096, 4, 1), (16, 32, 8, 128, 65536, 4096, 4, 0), (1, 4, 2, 64, 100, 8, 0, 0)):
-        ns = swaa.decode_num_splits(*args)
-        assert ns >= 1
+    for args in ((16, 32, 8, 128, 65536, 4096, 4, 1), (16, 32, 8, 128, 65536, 4096, 4, 0), (1, 4, 2, 64, 100, 8, 0, 0),
+                 (2, 64, 4, 128, 9000, 1, 0, 1)):
+        nb = swaa.decode_num_blocks(*args)
+        assert nb >= 1
         B, Hq, Hkv, D = args[:4]
-        assert swaa.decode_workspace_size(*args) >= B * Hq * ns * (D + 2) * 4
+        heads = 8 if Hq // Hkv <= 8 else 16
+        # one ticket per block and two partial slots per block, each (max, sum, O[D]) per head of a chunk
+        assert swaa.decode_workspace_size(*args) >= 4 * nb + 2 * nb * heads * (D + 2) * 4
+    # a problem of a single tile needs a single block
+    assert swaa.decode_num_blocks(1, 4, 2, 64, 100, 8, 0, 0) == 1

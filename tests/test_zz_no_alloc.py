@@ -2,7 +2,7 @@
 
 Some users of this library run attention at a point where they may not call cudaMalloc (a serving hot
 path, a plug-in without access to the host framework's memory pool, a process whose device memory is
-fully handed out).  For them the library carries its split-K scratch in a fixed 16 MiB array of its own.
+fully handed out).  For them the library carries its split-K scratch in a fixed 2 MiB array of its own.
 This test calls that entry point through the C ABI twice in a row, with different shapes and masks so
 that the second call finds the first call's leftovers in the shared array, and checks each result
 against swaa_decode with a caller-owned workspace.  It is collected last on purpose.
@@ -35,13 +35,13 @@ def _close(a, b):
 
 def test_decode_static_matches_decode_on_two_calls_in_a_row():
     calls = [
-        # first call: many splits, full attention; second: other shape, SWA mask, ragged lengths
+        # first call: sequences cut over many blocks, full attention; second: other shape, SWA mask, ragged lengths
         (inputs.DecodeConfig("a", 4, 20000, 32, 8, 128, 0, 0, seed=71, seqlens=(20000, 4101, 9000, 1)), 1, 0, True),
         (inputs.DecodeConfig("b", 3, 12000, 16, 2, 64, 0, 0, seed=72, seqlens=(12000, 5000, 300)), 4096, 4, False),
     ]
     for cfg, W, S, full in calls:
         q, kc, vc, sl = inputs.make_decode_inputs(cfg, "cuda")
-        assert swaa.decode_num_splits(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.Lmax, W, S, full) > 1
+        assert swaa.decode_num_blocks(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.Lmax, W, S, full) > 1
         want = _reference(q, kc, vc, sl, W, S, full)
         got = torch.full_like(q, float("nan"))
         before = torch.cuda.memory_allocated()
@@ -52,7 +52,7 @@ def test_decode_static_matches_decode_on_two_calls_in_a_row():
 
 
 def test_decode_static_rejects_shapes_beyond_its_scratch():
-    B, Lmax, Hq, Hkv, D = 64, 65536, 64, 8, 128
+    B, Lmax, Hq, Hkv, D = 64, 65536, 64, 4, 128  # 16 query heads per kv head: the largest partial buffers
     assert swaa.decode_workspace_size(B, Hq, Hkv, D, Lmax, 1, 0, True) > swaa.DECODE_STATIC_SCRATCH_BYTES
     q = torch.zeros((B, Hq, D), dtype=torch.bfloat16, device="cuda")
     kc = torch.zeros((B, 1, Hkv, D), dtype=torch.bfloat16, device="cuda")
