@@ -117,7 +117,7 @@ int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out
  *   - The first call on each device looks up the array's device address (once per device, with that
  *     device current) before it launches.  Make that first call outside any stream capture.
  *   - All calls on one device share the one array, and it keeps whatever the previous call left
- *     there; each call clears the part that must start at zero.  Two calls whose kernels can overlap
+ *     there; no part of it has to start at zero (tickets carry a per-call stamp).  Two calls whose kernels can overlap
  *     on the same GPU (different streams, no dependency between them) race on it: serialise them.
  * Returns the same status codes as swaa_decode.
  */

@@ -12,11 +12,13 @@
 // [c * tpc, (c+1) * tpc) of it, so every SM streams the same number of bytes whatever the batch
 // shape.  A block therefore holds at most two incomplete items (the first and the last of its run);
 // it writes complete items straight to `out` and incomplete ones as (max, sum, unnormalised O)
-// partials, which the last block to finish an item merges (atomic ticket, same launch).
+// partials, which the last block to finish an item merges (atomic ticket, same launch).  A ticket
+// carries a per-call stamp, so stale workspace contents are recognised and nothing has to be cleared.
 //
 // Data path.  One producer thread keeps a ring of shared-memory stages full with TMA tile copies
-// (K and V boxes of [64 keys][64 channels], 128-byte swizzle), so that the bytes in flight per SM do
-// not depend on registers or occupancy.  Four consumer warps each take 16 keys of every tile and run
+// (K and V boxes of [64 keys][64 channels], 128-byte swizzle; a 16-key box for tiles with at most 16
+// visible keys, e.g. the sinks), so that the bytes in flight per SM do not depend on registers or
+// occupancy.  Four consumer warps each take 16 keys of every tile and run
 // both contractions on warp-level tensor-core MMAs with fp32 accumulation in the transposed form
 //     S^T[16 keys x 8 heads] = K[16 keys x D] * Q^T[D x 8 heads]
 //     O^T[16 ch  x 8 heads] += V^T[16 ch x 16 keys] * P^T[16 keys x 8 heads]
@@ -41,15 +43,18 @@ struct DecodeParams {
     int IPB;       // items per sequence = Hkv * HG
     int window, n_sink, is_full;
     float sl2;     // softmax scale * log2(e)
-    int* tickets;  // [gridDim.x], zeroed before the launch
+    unsigned long long* tickets;  // [gridDim.x]; (call stamp << 16 | arrivals), needs no initialisation
+    unsigned long long stamp;     // 48-bit number unique to this call (never 0)
     float* part;   // [2 * gridDim.x][8*NH][D + 2]: per head (max in score units, sum, unnormalised O)
 };
 
 constexpr int kDecodeTileKeys = 64;
+constexpr int kDecodeSmallBoxKeys = 16;  // second TMA box for tiles with few visible keys
 constexpr int kDecodeConsumerWarps = 4;
 constexpr int kDecodeConsumerThreads = kDecodeConsumerWarps * 32;
 constexpr int kDecodeThreads = kDecodeConsumerThreads + 32;  // + the producer warp
 constexpr int kDecodeMinTilesPerBlock = 4;                   // do not cut the list finer than 256 keys
+constexpr int kDecodeWarpScanMaxB = 1024;                    // batches up to this size: warp-local scan
 
 template <int D, int NH>
 struct DecodeSmem {
@@ -136,9 +141,18 @@ __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumerThreads) : "memory");
 }
 
+#ifdef SWAA_DECODE_TIMING
+// Development aid: per-block time stamps (ns) of the phases of one launch.
+__device__ unsigned long long g_decode_stamps[256][8];
+#define SWAA_DSTAMP(slot) do { if ((threadIdx.x & 31) == 0 && blockIdx.x < 256) g_decode_stamps[blockIdx.x][slot] = global_timer_ns(); } while (0)
+#else
+#define SWAA_DSTAMP(slot)
+#endif
+
 template <int D, int NH>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
-decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const DecodeParams p) {
+decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+              const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16, const DecodeParams p) {
     static_assert(D == 64 || D == 128, "head size");
     using L = DecodeSmem<D, NH>;
     constexpr int ST = L::kStages;
@@ -164,49 +178,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ncta = (int)gridDim.x, cta = (int)blockIdx.x;
+    if (warp == 0) SWAA_DSTAMP(0);  // block entered
 
-    // ---- where does this block's run of the global tile list start?  (scan of tiles per sequence)
-    const int chunk = (p.B + kDecodeThreads - 1) / kDecodeThreads;
-    const int bb = min(p.B, tid * chunk), be = min(p.B, bb + chunk);
-    long long mine = 0;
-    for (int b = bb; b < be; ++b) {
-        const SeqGeom g = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
-        if (g.nt == 0) {
-            record_device_error(SWAA_ERR_BAD_SEQLENS);
-            if (b % ncta == cta) {  // this sequence has no tiles: its output rows are zero-filled here
-                uint4* o = reinterpret_cast<uint4*>(p.out + (size_t)b * p.Hq * D);
-                for (int i = 0; i < p.Hq * D / 8; ++i) o[i] = make_uint4(0, 0, 0, 0);
-            }
-        }
-        mine += (long long)g.nt * p.IPB;
-    }
-    sc_scan[tid] = mine;
-    __syncthreads();
-    for (int off = 1; off < kDecodeThreads; off <<= 1) {
-        const long long v = tid >= off ? sc_scan[tid - off] : 0;
-        __syncthreads();
-        sc_scan[tid] += v;
-        __syncthreads();
-    }
-    const long long total = sc_scan[kDecodeThreads - 1];
-    long long tpc = (total + ncta - 1) / ncta;
-    if (tpc < kDecodeMinTilesPerBlock) tpc = kDecodeMinTilesPerBlock;
-    const long long t0 = (long long)cta * tpc;
-    const long long t1 = total < t0 + tpc ? total : t0 + tpc;
-    if (t0 >= t1) return;  // nothing for this block (uniform: no barrier is pending)
-    if (sc_scan[tid] - mine <= t0 && t0 < sc_scan[tid]) {
-        long long acc = sc_scan[tid] - mine;
-        for (int b = bb; b < be; ++b) {
-            const SeqGeom g = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
-            const long long nb = (long long)g.nt * p.IPB;
-            if (t0 < acc + nb) {
-                sc_b0 = b;
-                sc_off = t0 - acc;
-                break;
-            }
-            acc += nb;
-        }
-    }
     if (tid == 0) {
         *abort_flag = 0;
         *sm_last = 0;
@@ -217,10 +190,108 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
+    if (tid == kDecodeConsumerThreads) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k16)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v16)) : "memory");
+    }
+
+    // ---- where does this block's run of the global tile list start?  (scan of tiles per sequence)
+    auto tiles_of = [&](int b) -> long long {
+        return (long long)decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full).nt * p.IPB;
+    };
+    auto zero_fill_bad = [&](int b) {  // a sequence without tiles: report it, zero its output rows (one block does)
+        record_device_error(SWAA_ERR_BAD_SEQLENS);
+        if (b % ncta == cta) {
+            uint4* o = reinterpret_cast<uint4*>(p.out + (size_t)b * p.Hq * D);
+            for (int i = 0; i < p.Hq * D / 8; ++i) o[i] = make_uint4(0, 0, 0, 0);
+        }
+    };
+    long long total, tpc, t0, t1, off0 = 0;
+    int b0 = 0;
+    if (p.B <= kDecodeWarpScanMaxB) {
+        // small batch: every warp scans all sequences by itself with shuffles, no block-level exchange
+        total = 0;
+        for (int base = 0; base < p.B; base += 32) {
+            const int b = base + lane;
+            long long nb = 0;
+            if (b < p.B) {
+                nb = tiles_of(b);
+                if (nb == 0 && warp == 0) zero_fill_bad(b);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) nb += __shfl_xor_sync(0xffffffffu, nb, o);
+            total += nb;
+        }
+        tpc = (total + ncta - 1) / ncta;
+        if (tpc < kDecodeMinTilesPerBlock) tpc = kDecodeMinTilesPerBlock;
+        t0 = (long long)cta * tpc;
+        t1 = total < t0 + tpc ? total : t0 + tpc;
+        if (t0 < t1) {
+            long long run = 0;
+            for (int base = 0; base < p.B; base += 32) {
+                const int b = base + lane;
+                const long long nb = b < p.B ? tiles_of(b) : 0;
+                long long incl = nb;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const long long v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                const bool here = run + incl - nb <= t0 && t0 < run + incl;
+                const unsigned hit = __ballot_sync(0xffffffffu, here);
+                if (hit) {
+                    const int src = __ffs(hit) - 1;
+                    b0 = base + src;
+                    off0 = t0 - (run + __shfl_sync(0xffffffffu, incl - nb, src));
+                    break;
+                }
+                run += __shfl_sync(0xffffffffu, incl, 31);
+            }
+        }
+        __syncthreads();  // barrier initialisation
+    } else {
+        const int chunk = (p.B + kDecodeThreads - 1) / kDecodeThreads;
+        const int bb = min(p.B, tid * chunk), be = min(p.B, bb + chunk);
+        long long mine = 0;
+        for (int b = bb; b < be; ++b) {
+            const long long nb = tiles_of(b);
+            if (nb == 0) zero_fill_bad(b);
+            mine += nb;
+        }
+        sc_scan[tid] = mine;
+        __syncthreads();
+        for (int off = 1; off < kDecodeThreads; off <<= 1) {
+            const long long v = tid >= off ? sc_scan[tid - off] : 0;
+            __syncthreads();
+            sc_scan[tid] += v;
+            __syncthreads();
+        }
+        total = sc_scan[kDecodeThreads - 1];
+        tpc = (total + ncta - 1) / ncta;
+        if (tpc < kDecodeMinTilesPerBlock) tpc = kDecodeMinTilesPerBlock;
+        t0 = (long long)cta * tpc;
+        t1 = total < t0 + tpc ? total : t0 + tpc;
+        if (t0 < t1 && sc_scan[tid] - mine <= t0 && t0 < sc_scan[tid]) {
+            long long acc = sc_scan[tid] - mine;
+            for (int b = bb; b < be; ++b) {
+                const long long nb = tiles_of(b);
+                if (t0 < acc + nb) {
+                    sc_b0 = b;
+                    sc_off = t0 - acc;
+                    break;
+                }
+                acc += nb;
+            }
+        }
+        __syncthreads();
+        b0 = sc_b0;
+        off0 = sc_off;
+    }
+    if (t0 >= t1) return;  // nothing for this block (uniform; nobody waits on a barrier)
+    if (warp == 0) SWAA_DSTAMP(1);  // start position known
     const int cnt = (int)(t1 - t0);  // tpc <= tiles of the whole problem / blocks, far below 2^31 in practice
-    const int b0 = sc_b0;
-    const long long off0 = sc_off;
 
     if (warp == kDecodeConsumerWarps) {
         // =========================================================================== TMA producer
@@ -235,14 +306,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 if (!ok) break;
                 const int key0 = w.key0(), hk = w.hv / p.HG;
                 const uint32_t dst = smem_base + (uint32_t)s * L::kStageBytes;
-                mbar_arrive_expect_tx(bar_kf(s), (uint32_t)L::kTileBytes);
+                // a tile with at most 16 visible keys (typically the sinks) is fetched with the 16-row box
+                const bool small = w.valid() <= kDecodeSmallBoxKeys;
+                const CUtensorMap* mk = small ? &tm_k16 : &tm_k;
+                const CUtensorMap* mv = small ? &tm_v16 : &tm_v;
+                const uint32_t bytes = small ? (uint32_t)(L::kPanels * kDecodeSmallBoxKeys * 128) : (uint32_t)L::kTileBytes;
+                mbar_arrive_expect_tx(bar_kf(s), bytes);
 #pragma unroll
                 for (int pn = 0; pn < L::kPanels; ++pn)
-                    tma_load_4d(dst + pn * L::kPanelBytes, &tm_k, pn * 64, hk, key0, w.b, bar_kf(s));
-                mbar_arrive_expect_tx(bar_vf(s), (uint32_t)L::kTileBytes);
+                    tma_load_4d(dst + pn * L::kPanelBytes, mk, pn * 64, hk, key0, w.b, bar_kf(s));
+                mbar_arrive_expect_tx(bar_vf(s), bytes);
 #pragma unroll
                 for (int pn = 0; pn < L::kPanels; ++pn)
-                    tma_load_4d(dst + L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, key0, w.b, bar_vf(s));
+                    tma_load_4d(dst + L::kTileBytes + pn * L::kPanelBytes, mv, pn * 64, hk, key0, w.b, bar_vf(s));
                 if (++s == ST) {
                     s = 0;
                     ph ^= 1u;
@@ -314,6 +390,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             const int vw = w.valid() - 16 * warp;  // visible keys among this warp's 16
             const uint32_t stage = smem_base + (uint32_t)s * L::kStageBytes;
             ok = ok && mbar_wait(bar_kf(s), ph, abort_flag);
+            if (warp == 0 && n == 0) SWAA_DSTAMP(2);  // first K tile landed
             if (ok && vw > 0) {
                 // ---- S^T = K Q^T : rows = keys (g, g+8), cols = heads (2c, 2c+1)
                 float sacc[NH][4];
@@ -403,6 +480,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
 
         // ---- merge the four warps of the block through shared memory
+        if (warp == 0 && n == cnt) SWAA_DSTAMP(3);  // last tile consumed
 #pragma unroll
         for (int nh = 0; nh < NH; ++nh) {
 #pragma unroll
@@ -460,8 +538,17 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             __threadfence();
             consumer_sync();
             if (tid == 0) {
-                const int ticket = atomicAdd(&p.tickets[c_first], 1);
-                *sm_last = (ticket == c_last - c_first) ? 1 : 0;
+                // A ticket whose stamp is not this call's is left over from an earlier call (or was never
+                // written): the first block to arrive restarts it, so the workspace needs no clearing.
+                unsigned long long* t = p.tickets + c_first;
+                unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(t), want;
+                for (;;) {
+                    want = (seen >> 16) == p.stamp ? seen + 1ull : ((p.stamp << 16) | 1ull);
+                    const unsigned long long prev = atomicCAS(t, seen, want);
+                    if (prev == seen) break;
+                    seen = prev;
+                }
+                *sm_last = ((int)(want & 0xffffull) == c_last - c_first + 1) ? 1 : 0;
             }
             consumer_sync();
             if (*sm_last && ok) {
@@ -490,6 +577,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         consumer_sync();  // the merge buffers are free for the next segment
         first_seg = false;
     }
+    if (warp == 0) SWAA_DSTAMP(4);  // done
 }
 
 }  // namespace swaa

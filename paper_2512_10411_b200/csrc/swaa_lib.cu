@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include <mutex>
+#include <random>
 
 #include "swaa.h"
 #include "swaa_internal.cuh"
@@ -46,6 +47,7 @@ struct DecodePlan {
     int NH;      // 8-head blocks per chunk (1 or 2)
     int HG;      // chunks per kv head
     int blocks;  // persistent grid size
+    bool too_large;
     size_t off_part, bytes;
 };
 
@@ -66,9 +68,21 @@ static DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int Lmax, int windo
     if (blocks > sms) blocks = sms;
     if (blocks < 1) blocks = 1;
     pl.blocks = (int)blocks;
-    pl.off_part = ((size_t)pl.blocks * sizeof(int) + 255) / 256 * 256;
+    pl.too_large = tiles_ub / blocks > 0x3fffffffLL;  // the kernel counts a block's tiles in an int
+    pl.off_part = ((size_t)pl.blocks * sizeof(unsigned long long) + 255) / 256 * 256;
     pl.bytes = pl.off_part + (size_t)2 * pl.blocks * HC * (D + 2) * sizeof(float);
     return pl;
+}
+
+// 48-bit stamps, unique per call within the process and never 0.  They start at a random point so that
+// what an earlier process or an unrelated buffer left in a workspace does not look like a live ticket.
+static unsigned long long next_call_stamp() {
+    static std::atomic<unsigned long long> counter{[] {
+        std::random_device rd;
+        const unsigned long long r = ((unsigned long long)rd() << 32) ^ (unsigned long long)rd();
+        return (r & 0x3fffffffffffull) | 0x400000000000ull;  // in [2^46, 2^47)
+    }()};
+    return counter.fetch_add(1, std::memory_order_relaxed) & 0xffffffffffffull;
 }
 
 static int check_decode_shape(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full) {
@@ -99,14 +113,14 @@ static EncodeTiledFn encode_tiled_fn() {
 }
 
 // Tensor map over a bf16 cache [B, Lmax, Hkv, D]: dimensions (D, Hkv, Lmax, B) innermost first; one box
-// is [64 entries] x [1 head] x [64 channels] = 64 rows of 128 bytes, written with the 128-byte swizzle.
+// is [box_keys entries] x [1 head] x [64 channels] = rows of 128 bytes, written with the 128-byte swizzle.
 // Rows past Lmax are filled with zeros.
-static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, int Hkv, int D) {
+static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, int Hkv, int D, int box_keys) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return SWAA_ERR_CUDA;
     const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)Lmax, (cuuint64_t)B};
     const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)Hkv * D * 2, (cuuint64_t)Lmax * Hkv * D * 2};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)kDecodeTileKeys, 1};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_keys, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -115,13 +129,12 @@ static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, i
 }
 
 template <int D, int NH>
-static int launch_decode(const CUtensorMap& tk, const CUtensorMap& tv, const DecodeParams& p, int blocks,
-                         cudaStream_t st) {
+static int launch_decode(const CUtensorMap (&tm)[4], const DecodeParams& p, int blocks, cudaStream_t st) {
     using L = DecodeSmem<D, NH>;
     if (cudaFuncSetAttribute(decode_kernel<D, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
         cudaSuccess)
         return SWAA_ERR_CUDA;
-    decode_kernel<D, NH><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tk, tv, p);
+    decode_kernel<D, NH><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tm[0], tm[1], tm[2], tm[3], p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
@@ -160,12 +173,15 @@ extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache
     if (rc != SWAA_OK) return rc;
     if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
     const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count);
+    if (pl.too_large) return SWAA_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < pl.bytes)
         return SWAA_ERR_WORKSPACE;
 
-    CUtensorMap tk, tv;
-    if ((rc = make_cache_map(&tk, kcache, B, Lmax, Hkv, D)) != SWAA_OK) return rc;
-    if ((rc = make_cache_map(&tv, vcache, B, Lmax, Hkv, D)) != SWAA_OK) return rc;
+    CUtensorMap tm[4];  // K, V with the full box; K, V with the small box
+    if ((rc = make_cache_map(&tm[0], kcache, B, Lmax, Hkv, D, kDecodeTileKeys)) != SWAA_OK) return rc;
+    if ((rc = make_cache_map(&tm[1], vcache, B, Lmax, Hkv, D, kDecodeTileKeys)) != SWAA_OK) return rc;
+    if ((rc = make_cache_map(&tm[2], kcache, B, Lmax, Hkv, D, kDecodeSmallBoxKeys)) != SWAA_OK) return rc;
+    if ((rc = make_cache_map(&tm[3], vcache, B, Lmax, Hkv, D, kDecodeSmallBoxKeys)) != SWAA_OK) return rc;
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     DecodeParams p;
@@ -185,14 +201,12 @@ extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache
     const float sc = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
     p.sl2 = sc * 1.4426950408889634f;
     char* ws = static_cast<char*>(workspace);
-    p.tickets = reinterpret_cast<int*>(ws);
+    p.tickets = reinterpret_cast<unsigned long long*>(ws);
     p.part = reinterpret_cast<float*>(ws + pl.off_part);
-    if (pl.blocks > 1) {
-        if (cudaMemsetAsync(p.tickets, 0, pl.off_part, st) != cudaSuccess) return SWAA_ERR_CUDA;
-    }
+    p.stamp = next_call_stamp();
     if (D == 128)
-        return pl.NH == 1 ? launch_decode<128, 1>(tk, tv, p, pl.blocks, st) : launch_decode<128, 2>(tk, tv, p, pl.blocks, st);
-    return pl.NH == 1 ? launch_decode<64, 1>(tk, tv, p, pl.blocks, st) : launch_decode<64, 2>(tk, tv, p, pl.blocks, st);
+        return pl.NH == 1 ? launch_decode<128, 1>(tm, p, pl.blocks, st) : launch_decode<128, 2>(tm, p, pl.blocks, st);
+    return pl.NH == 1 ? launch_decode<64, 1>(tm, p, pl.blocks, st) : launch_decode<64, 2>(tm, p, pl.blocks, st);
 }
 
 // ----------------------------------------------------------------------------------------- prefill
@@ -321,8 +335,8 @@ extern "C" int swaa_decode_static(const void* q, const void* kcache, const void*
     void* scratch = nullptr;
     const int rs = decode_static_scratch(&scratch);
     if (rs != SWAA_OK) return rs;
-    // Same kernel and same plan as swaa_decode; its tickets (the only part that must start at zero) are
-    // cleared by that call on `stream` before the kernel runs.
+    // Same kernel and same plan as swaa_decode.  Nothing in the scratch has to start at zero: tickets are
+    // stamped per call, partial results are written before they are read.
     return swaa_decode(q, kcache, vcache, out, seqlens, B, Lmax, Hq, Hkv, D, window, n_sink, is_full, scale, scratch,
                        SWAA_DECODE_STATIC_SCRATCH_BYTES, stream);
 }
@@ -400,6 +414,15 @@ extern "C" int swaa_last_device_status(void* stream) {
     }
     return value;
 }
+
+#ifdef SWAA_DECODE_TIMING
+extern "C" int swaa_debug_read_decode_stamps(unsigned long long* out, int n_blocks) {
+    if (n_blocks > 256) n_blocks = 256;
+    if (cudaMemcpyFromSymbol(out, g_decode_stamps, sizeof(unsigned long long) * 8 * n_blocks) != cudaSuccess)
+        return SWAA_ERR_CUDA;
+    return SWAA_OK;
+}
+#endif
 
 #ifdef SWAA_PHASE_TIMING
 extern "C" int swaa_debug_read_phases(unsigned long long* out32, int reset) {

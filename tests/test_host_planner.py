@@ -122,6 +122,6 @@ def test_decode_split_plan_is_consistent():
         B, Hq, Hkv, D = args[:4]
         heads = 8 if Hq // Hkv <= 8 else 16
         # one ticket per block and two partial slots per block, each (max, sum, O[D]) per head of a chunk
-        assert swaa.decode_workspace_size(*args) >= 4 * nb + 2 * nb * heads * (D + 2) * 4
+        assert swaa.decode_workspace_size(*args) >= 8 * nb + 2 * nb * heads * (D + 2) * 4
     # a problem of a single tile needs a single block
     assert swaa.decode_num_blocks(1, 4, 2, 64, 100, 8, 0, 0) == 1
