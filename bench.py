@@ -35,7 +35,7 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists).
-PREFILL_DRAM_TRAFFIC_BYTES = None
+PREFILL_DRAM_TRAFFIC_BYTES = 643980800  # 405.03 MB read + 238.95 MB written, profiles/prefill_kernel_cfg2_long_swa.txt
 
 
 def visible_pairs(L, W, S, full):
