@@ -37,6 +37,10 @@ L2_FLUSH_BYTES = 256 << 20
 # summarised under profiles/ (None until a capture exists).
 PREFILL_DRAM_TRAFFIC_BYTES = 643980800  # 405.03 MB read + 238.95 MB written, profiles/prefill_kernel_cfg2_long_swa.txt
 
+# decode kernel: 4 x (1.0739 GB read + 4 MB written) scaled from the B=4 capture; 270.0 MB + 5 MB at full size
+DECODE_FA_DRAM_TRAFFIC_BYTES = 4 * (1073919000 + 4249600)
+DECODE_SWA_DRAM_TRAFFIC_BYTES = 269955584 + 4963840
+
 
 def visible_pairs(L, W, S, full):
     if full or W >= L:
@@ -349,11 +353,13 @@ def run_ours(args, rank, local_rank, world):
         "decode": {
             "fa": {"gbs": N * fa_gbs, "us_per_launch": 1e3 * t_fa / K, "bytes": fa_bytes,
                    "roofline": {"bound": "hbm", "achieved": fa_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                "frac": fa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": fa_gbs / 8000.0},
+                                "frac": fa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": fa_gbs / 8000.0,
+                                "traffic": DECODE_FA_DRAM_TRAFFIC_BYTES},
                    "e2e_gbs": fa_bytes / (e2e_fa_ms * 1e-3) / 1e9},
             "swa": {"gbs": N * swa_gbs, "us_per_launch": 1e3 * t_swa / K, "bytes": swa_bytes,
                     "roofline": {"bound": "hbm", "achieved": swa_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                 "frac": swa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": swa_gbs / 8000.0},
+                                 "frac": swa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": swa_gbs / 8000.0,
+                                 "traffic": DECODE_SWA_DRAM_TRAFFIC_BYTES},
                     "e2e_gbs": swa_bytes / (e2e_swa_ms * 1e-3) / 1e9},
         },
         "cpu_baseline": cpu_baseline,
@@ -392,6 +398,74 @@ def run_profile_case(case: str):
     print(json.dumps({"profile_case": case, "launches": swaa.kernel_launch_count()}))
 
 
+def run_sweep():
+    """Times swaa_prefill on the other workloads and on the parameter sweeps that show how the time depends
+    on L, W and n_sink (one GPU; median of a few launches, L2 flushed before each; one JSON line per case)."""
+    import dataclasses
+
+    import torch
+
+    import paper_2512_10411_b200 as swaa
+    from paper_2512_10411_b200 import inputs
+
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    flush_rd = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def time_case(tag, cfg, is_full, reps=5, tensors=None):
+        q, k, v, cu = tensors if tensors is not None else inputs.make_prefill_inputs(cfg, "cuda")
+        out = torch.empty_like(q)
+        ms = []
+        for r in range(reps + 1):
+            flush.zero_()
+            flush_rd.sum()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            swaa.swaa_prefill(q, k, v, out, cu, max(cfg.seqlens), cfg.window, cfg.n_sink, is_full)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if r > 0:
+                ms.append(a.elapsed_time(b))
+        assert swaa.last_device_status() == 0
+        ms.sort()
+        med = ms[len(ms) // 2]
+        pairs = sum(visible_pairs(L, cfg.window, cfg.n_sink, is_full) for L in cfg.seqlens)
+        flops = 4.0 * cfg.D * cfg.Hq * pairs
+        tf = flops / (med * 1e-3) / 1e12
+        line = {"case": tag, "seqlens": list(cfg.seqlens) if len(cfg.seqlens) > 1 else cfg.seqlens[0], "Hq": cfg.Hq,
+                "Hkv": cfg.Hkv, "D": cfg.D, "window": cfg.window, "n_sink": cfg.n_sink, "is_full": bool(is_full),
+                "ms": med, "ms_min": ms[0], "effective_tflops": tf, "frac_of_measured_peak": tf / peaks["bf16_tflops"],
+                "frac_of_nominal_2250": tf / 2250.0, "us_per_1k_tokens": 1e3 * med / (sum(cfg.seqlens) / 1024.0)}
+        print(json.dumps(line), flush=True)
+        del out
+        return med
+
+    # time against L at fixed W (App. A: O(N*W)), then the sink and window variants on workload 2
+    for L in (8192, 16384, 32768, 65536, 131072):
+        time_case("linear_in_L", inputs.cfg_long(L=L), False)
+    for S in (0, 4, 100):
+        time_case("sinks", inputs.cfg_long(n_sink=S), False)
+    for W in (1024, 2048, 4096, 8192):
+        time_case("window", inputs.cfg_long(window=W), False)
+    time_case("cfg2_full_causal", inputs.cfg_long(is_full=True), True, reps=3)
+    time_case("cfg5_varlen", inputs.cfg_varlen(), False, reps=3)
+    time_case("cfg1_tiny", inputs.cfg_tiny(), False)
+    # workload 3: the 36-layer interleaved stack, per layer and in total (mask policy from the layer schedule)
+    pol = swaa.SwaaPolicy(n_layers=36, window=4096, n_sink=64, fa_start=3, fa_step=4, fa_decode=True)
+    total, per_kind = 0.0, {False: [], True: []}
+    for layer in range(pol.n_layers):
+        cfg = inputs.cfg_stack_layer(layer)
+        full = swaa.schedule_is_full(pol, layer, 0)
+        t = time_case(f"cfg3_layer{layer:02d}", cfg, full, reps=1)
+        total += t
+        per_kind[bool(full)].append(t)
+    print(json.dumps({"case": "cfg3_stack_total", "layers": pol.n_layers, "ms_total": total,
+                      "swa_layers": len(per_kind[False]), "ms_per_swa_layer": sum(per_kind[False]) / len(per_kind[False]),
+                      "fa_layers": len(per_kind[True]), "ms_per_fa_layer": sum(per_kind[True]) / len(per_kind[True])}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -402,7 +476,12 @@ def main():
                     choices=["prefill", "prefill_full", "prefill_tiny", "decode_fa", "decode_swa", "decode_fa_small",
                              "decode_swa_small"],
                     help="run three launches of one kernel only (for ncu) and exit")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time swaa_prefill on the other workloads and the L / W / n_sink sweeps (one GPU) and exit")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep()
+        return
     if args.profile_case:
         run_profile_case(args.profile_case)
         return
