@@ -78,6 +78,27 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         : "memory");
 }
 
+// The same with the shared-memory descriptors given as (low word, shared high word): the low word holds
+// the start address and the leading-dimension offset, so stepping through a tile is one 32-bit add per operand.
+__device__ __forceinline__ void mma_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // Packed pairs of fp32 in one 64-bit register (two lanes per FMA/ADD instruction on sm_100).
 __device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
     uint64_t r;
@@ -102,6 +123,34 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+
+// 2^x for a pair of arguments on the FMA and integer pipes instead of the special-function unit:
+// x = n + f with n = round(x), f in [-1/2, 1/2]; 2^f by a cubic (relative error 7.6e-5, far below the
+// bf16 rounding of P); n is added into the exponent field.  Arguments below -126 (masked scores arrive
+// as -inf) give exactly 0, as ex2.approx.ftz does.
+__device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, float& r1) {
+    const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    const uint64_t xx = pack_f32x2(x0, x1);
+    uint64_t t, fl, f, q;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(t) : "l"(xx), "l"(pack_f32x2(kMagic, kMagic)));
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(fl) : "l"(t), "l"(pack_f32x2(kMagic, kMagic)));
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(f) : "l"(xx), "l"(fl));
+    q = fma_f32x2(f, pack_f32x2(0.05520550534129143f, 0.05520550534129143f),
+                  pack_f32x2(0.24261397123336792f, 0.24261397123336792f));
+    q = fma_f32x2(q, f, pack_f32x2(0.6932547688484192f, 0.6932547688484192f));
+    q = fma_f32x2(q, f, pack_f32x2(0.9999276995658875f, 0.9999276995658875f));
+    float t0, t1, q0, q1;
+    unpack_f32x2(t, t0, t1);
+    unpack_f32x2(q, q0, q1);
+    r0 = x0 < -126.f ? 0.f : __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    r1 = x1 < -126.f ? 0.f : __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
+// Bit c (0..15) set: column pair c of every 32-column chunk of a score tile takes the polynomial path.
+#ifndef SWAA_POLY_PAIR_MASK
+#define SWAA_POLY_PAIR_MASK 0x8888u
+#endif
+constexpr uint32_t kPolyPairMask = SWAA_POLY_PAIR_MASK;
 
 #define SWAA_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
 #define SWAA_I8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
@@ -365,23 +414,39 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (lane == 0) {
             const uint32_t tS[2] = {tmem_base, tmem_base + 128u};
             const uint32_t tO[2] = {tmem_base + 256u, tmem_base + 256u + (uint32_t)D};
+            // Descriptor words are built once: per operand tile a low word (address, leading-dimension offset)
+            // and one shared high word (stride 1024 B, descriptor version, 128-byte swizzle).  The issue latency
+            // of this thread is part of every tile's critical path, so the per-MMA work is one add per operand.
+            const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0, 0, 1024) >> 32);
+            uint32_t q_lo[2], k_lo[ST], v_lo[ST];
+#pragma unroll
+            for (int sd = 0; sd < 2; ++sd) q_lo[sd] = (uint32_t)smem_desc_sw128(sQ + sd * L::kTileBytes, 16, 1024);
+#pragma unroll
+            for (int st = 0; st < ST; ++st) {
+                k_lo[st] = (uint32_t)smem_desc_sw128(sK + st * L::kTileBytes, 16, 1024);
+                v_lo[st] = (uint32_t)smem_desc_sw128(sV + st * L::kTileBytes, L::kPanelBytes, 1024);
+            }
+            auto pick = [&](const uint32_t (&arr)[ST], int stage) -> uint32_t {  // register array, static indices only
+                uint32_t r = arr[0];
+#pragma unroll
+                for (int st = 1; st < ST; ++st) r = stage == st ? arr[st] : r;
+                return r;
+            };
             auto issue_qk = [&](int side, int stage) {
-                const uint32_t qa = sQ + side * L::kTileBytes, kb = sK + stage * L::kTileBytes;
+                const uint32_t qa = side ? q_lo[1] : q_lo[0], kb = pick(k_lo, stage), d = tS[side];
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (uint32_t)(kk >> 2) * L::kPanelBytes + (uint32_t)(kk & 3) * 32u;
-                    mma_ss(tS[side], smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024),
-                           kIdescQK, kk > 0 ? 1u : 0u);
+                    const uint32_t off = ((uint32_t)(kk >> 2) * L::kPanelBytes + (uint32_t)(kk & 3) * 32u) >> 4;
+                    mma_ss_lh(d, qa + off, kb + off, desc_hi, kIdescQK, kk > 0 ? 1u : 0u);
                 }
             };
             auto issue_pv = [&](int side, int stage, bool acc) {
-                const uint32_t vb = sV + stage * L::kTileBytes;
+                const uint32_t vb = pick(v_lo, stage), d = tO[side], a = tS[side];
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk) {
                     // P: 16 keys = 8 TMEM columns of packed bf16 pairs.  V: 16 key rows of 128 bytes.
-                    mma_ts(tO[side], tS[side] + (uint32_t)kk * 8u,
-                           smem_desc_sw128(vb + (uint32_t)kk * 2048u, L::kPanelBytes, 1024), kIdescPV,
-                           (acc || kk > 0) ? 1u : 0u);
+                    mma_ts_lh(d, a + (uint32_t)kk * 8u, vb + (((uint32_t)kk * 2048u) >> 4), desc_hi, kIdescPV,
+                              (acc || kk > 0) ? 1u : 0u);
                 }
             };
             int g = 0;                 // K/V ring position
@@ -578,7 +643,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                             sl2x2, noffx2);
                         float x0, x1;
                         unpack_f32x2(x, x0, x1);
-                        const float p0 = ex2f(x0), p1 = ex2f(x1);
+                        float p0, p1;
+                        if ((kPolyPairMask >> c) & 1u) {
+                            exp2_poly_x2(x0, x1, p0, p1);  // FMA pipe: takes load off the special-function unit
+                        } else {
+                            p0 = ex2f(x0);
+                            p1 = ex2f(x1);
+                        }
                         if (c & 1) psum_b = add_f32x2(psum_b, pack_f32x2(p0, p1));
                         else psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
                         pk[c] = pack_bf16x2(p0, p1);
