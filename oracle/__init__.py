@@ -12,5 +12,6 @@ from .swaa_oracle import (  # noqa: F401
     layer_is_full,
     num_threads,
     prefill,
+    prefill_chunked,
     visible,
 )

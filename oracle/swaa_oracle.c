@@ -157,6 +157,55 @@ int swaa_oracle_prefill(const float* q, const float* k, const float* v, const in
 }
 
 /*
+ * Chunked prefill: the queries of sequence b are the LAST len_q tokens of a context of len_k >= len_q
+ * tokens whose keys and values are all given (Sec. 3.1.1 / Fig. 1a: later tokens attend to the stored
+ * context; a serving engine feeds a long prompt in chunks).  Query i of the chunk sits at position
+ * len_k - len_q + i of its sequence and sees the keys the mask policy allows for that position.
+ *   q [Tq, Hq, D] packed by cu_q [B+1]; k, v [Tk, Hkv, D] packed by cu_k [B+1]; float32 (bf16 values).
+ * Rows are chosen as in swaa_oracle_prefill, row_t being a packed QUERY token index.
+ * Returns 0, or -1 on inconsistent arguments (also len_q > len_k).
+ */
+int swaa_oracle_prefill_chunked(const float* q, const float* k, const float* v, const int32_t* cu_q,
+                                const int32_t* cu_k, int B, int Hq, int Hkv, int D, int64_t W, int64_t S,
+                                int is_full, double scale, int64_t n_rows, const int64_t* row_t,
+                                const int32_t* row_h, double* out, double* lse, double* psum, int64_t* nvis) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
+    if (!is_full && W < 1) return -1;
+    if (S < 0) return -1;
+    const int G = Hq / Hkv;
+    const int64_t Tq = B > 0 ? cu_q[B] : 0;
+    int64_t max_len = 0;
+    for (int b = 0; b < B; ++b) {
+        int64_t lq = (int64_t)cu_q[b + 1] - cu_q[b], lk = (int64_t)cu_k[b + 1] - cu_k[b];
+        if (lq < 0 || lk < lq) return -1;
+        if (lk > max_len) max_len = lk;
+    }
+    if (row_t == NULL && n_rows != Tq * Hq) return -1;
+    int bad = 0;
+#pragma omp parallel
+    {
+        double* scores = (double*)malloc(sizeof(double) * (size_t)(max_len > 0 ? max_len : 1));
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            int64_t t = row_t ? row_t[r] : r / Hq;
+            int h = row_t ? row_h[r] : (int)(r % Hq);
+            if (t < 0 || t >= Tq || h < 0 || h >= Hq) { bad = 1; continue; }
+            int b = 0;
+            while (!(cu_q[b] <= t && t < cu_q[b + 1])) ++b; /* sequence that owns query token t */
+            int64_t lq = (int64_t)cu_q[b + 1] - cu_q[b], lk = (int64_t)cu_k[b + 1] - cu_k[b];
+            int64_t i = (lk - lq) + (t - cu_q[b]); /* position of the query inside its sequence */
+            int64_t kstart = cu_k[b];
+            int hk = h / G;
+            oracle_row(q + (t * Hq + h) * (int64_t)D, k + (kstart * Hkv + hk) * (int64_t)D,
+                       v + (kstart * Hkv + hk) * (int64_t)D, i, (int64_t)Hkv * D, D, W, S, is_full, scale,
+                       out + r * D, lse ? lse + r : NULL, psum ? psum + r : NULL, nvis ? nvis + r : NULL, scores);
+        }
+        free(scores);
+    }
+    return bad ? -1 : 0;
+}
+
+/*
  * Decode: one query token per sequence against a dense cache.
  *   q [B, Hq, D]; kcache, vcache [B, Lmax, Hkv, D]; seqlens [B] counts the valid
  *   cache entries INCLUDING the current token, so the query's position is

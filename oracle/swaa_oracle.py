@@ -45,6 +45,9 @@ def _load():
         lib.swaa_oracle_prefill.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl, i64,
                                             vp, vp, vp, vp, vp, vp]
         lib.swaa_oracle_prefill.restype = ctypes.c_int
+        lib.swaa_oracle_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
+                                                    i64, vp, vp, vp, vp, vp, vp]
+        lib.swaa_oracle_prefill_chunked.restype = ctypes.c_int
         lib.swaa_oracle_decode.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
                                            vp, vp, vp, vp]
         lib.swaa_oracle_decode.restype = ctypes.c_int
@@ -114,6 +117,45 @@ def prefill(q, k, v, cu_seqlens, window: int, n_sink: int, is_full: bool, scale:
     if rows is None:
         return {"out": out.reshape(T, Hq, D), "lse": lse.reshape(T, Hq), "psum": psum.reshape(T, Hq),
                 "nvis": nvis.reshape(T, Hq)}
+    return {"out": out, "lse": lse, "psum": psum, "nvis": nvis}
+
+
+def prefill_chunked(q, k, v, cu_seqlens_q, cu_seqlens_k, window: int, n_sink: int, is_full: bool,
+                    scale: float | None = None, rows=None):
+    """Chunked prefill: queries are the last len_q tokens of each sequence's len_k-token context.
+
+    q [Tq,Hq,D] packed by cu_seqlens_q; k, v [Tk,Hkv,D] packed by cu_seqlens_k.  rows as in prefill()
+    (row_t indexes packed query tokens).  Returns a dict with out, lse, psum, nvis.
+    """
+    q, k, v = _f32(q), _f32(k), _f32(v)
+    Tq, Hq, D = q.shape
+    Tk, Hkv, _ = k.shape
+    assert k.shape == (Tk, Hkv, D) and v.shape == (Tk, Hkv, D)
+    cq = np.ascontiguousarray(np.asarray(cu_seqlens_q, dtype=np.int32))
+    ck = np.ascontiguousarray(np.asarray(cu_seqlens_k, dtype=np.int32))
+    B = cq.shape[0] - 1
+    assert ck.shape[0] == B + 1 and cq[0] == 0 and ck[0] == 0 and cq[-1] == Tq and ck[-1] == Tk
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    if rows is None:
+        n_rows, rt, rh = Tq * Hq, None, None
+    else:
+        rt = np.ascontiguousarray(np.asarray(rows[0], dtype=np.int64))
+        rh = np.ascontiguousarray(np.asarray(rows[1], dtype=np.int32))
+        n_rows = rt.shape[0]
+        assert rh.shape[0] == n_rows
+    out = np.empty((n_rows, D), dtype=np.float64)
+    lse = np.empty(n_rows, dtype=np.float64)
+    psum = np.empty(n_rows, dtype=np.float64)
+    nvis = np.empty(n_rows, dtype=np.int64)
+    rc = _load().swaa_oracle_prefill_chunked(_ptr(q), _ptr(k), _ptr(v), _ptr(cq), _ptr(ck), B, Hq, Hkv, D, int(window),
+                                             int(n_sink), int(bool(is_full)), float(scale), n_rows, _ptr(rt), _ptr(rh),
+                                             _ptr(out), _ptr(lse), _ptr(psum), _ptr(nvis))
+    if rc != 0:
+        raise ValueError("swaa_oracle_prefill_chunked: inconsistent arguments")
+    if rows is None:
+        return {"out": out.reshape(Tq, Hq, D), "lse": lse.reshape(Tq, Hq), "psum": psum.reshape(Tq, Hq),
+                "nvis": nvis.reshape(Tq, Hq)}
     return {"out": out, "lse": lse, "psum": psum, "nvis": nvis}
 
 

@@ -1,0 +1,106 @@
+"""Pins for the chunked-prefill oracle (queries = the last len_q tokens of a len_k-token context).  CPU only.
+
+What could go wrong and which test catches it: the position offset len_k - len_q dropped or applied with
+the wrong sign (numpy brute force, decode equivalence), keys taken from the wrong sequence of the
+packed key buffer (packed-batch test), sinks or window measured from the chunk instead of the
+sequence (numpy brute force with W and S smaller than the offset).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+
+def _bf16_randn(shape, seed):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randn(shape, generator=g).to(torch.bfloat16).to(torch.float32).numpy()
+
+
+def _visible_positions(pos, W, S, is_full):
+    """Keys a query at position `pos` sees, as a union of index ranges (window of W keys ending at the
+    query AND the first S tokens; Sec. 3.2.1), not as the oracle's predicate."""
+    if is_full:
+        return list(range(pos + 1))
+    return sorted(set(range(max(0, pos - W + 1), pos + 1)) | set(range(min(S, pos + 1))))
+
+
+def _numpy_rows(q, k, v, lq, lk, W, S, is_full, scale):
+    """Hand-written float64 softmax over the range-union key set, one sequence."""
+    Hq, Hkv = q.shape[1], k.shape[1]
+    G = Hq // Hkv
+    out = np.zeros((lq, Hq, q.shape[2]))
+    for i in range(lq):
+        keys = _visible_positions(lk - lq + i, W, S, is_full)
+        for h in range(Hq):
+            s = (k[keys, h // G].astype(np.float64) @ q[i, h].astype(np.float64)) * scale
+            p = np.exp(s - s.max())
+            out[i, h] = (p / p.sum()) @ v[keys, h // G].astype(np.float64)
+    return out
+
+
+@pytest.mark.parametrize("lq,lk", [(1, 1), (5, 5), (3, 40), (17, 64), (40, 41)])
+@pytest.mark.parametrize("W,S,full", [(1, 0, False), (8, 0, False), (8, 3, False), (5, 20, False), (100, 0, False), (1, 0, True)])
+def test_chunked_matches_numpy_bruteforce(lq, lk, W, S, full):
+    Hq, Hkv, D = 4, 2, 16
+    q, k, v = _bf16_randn((lq, Hq, D), 1), _bf16_randn((lk, Hkv, D), 2), _bf16_randn((lk, Hkv, D), 3)
+    r = oracle.prefill_chunked(q, k, v, [0, lq], [0, lk], W, S, full, scale=0.3)
+    want = _numpy_rows(q, k, v, lq, lk, W, S, full, 0.3)
+    assert np.allclose(r["out"], want, rtol=0, atol=1e-12)
+    assert np.allclose(r["psum"], 1.0, atol=1e-12)
+    for i in range(lq):
+        assert (r["nvis"][i] == len(_visible_positions(lk - lq + i, W, S, full))).all()
+
+
+def test_chunks_reproduce_the_one_shot_prefill():
+    """Feeding a prompt in chunks (each chunk's queries against the context so far) gives the rows of the
+    self-attention prefill of the whole prompt (Fig. 1a: later tokens attend to the stored context)."""
+    L, Hq, Hkv, D, W, S = 90, 4, 2, 16, 16, 3
+    q, k, v = _bf16_randn((L, Hq, D), 4), _bf16_randn((L, Hkv, D), 5), _bf16_randn((L, Hkv, D), 6)
+    whole = oracle.prefill(q, k, v, [0, L], W, S, False)
+    done = 0
+    for chunk in (7, 32, 1, 50):
+        end = done + chunk
+        r = oracle.prefill_chunked(q[done:end], k[:end], v[:end], [0, chunk], [0, end], W, S, False)
+        assert np.array_equal(r["out"], whole["out"][done:end])
+        assert np.array_equal(r["nvis"], whole["nvis"][done:end])
+        done = end
+    assert done == L
+
+
+def test_chunk_of_one_token_is_decode():
+    B, Lmax, Hq, Hkv, D = 3, 50, 4, 2, 16
+    sl = [50, 1, 23]
+    q = _bf16_randn((B, Hq, D), 7)
+    kc, vc = _bf16_randn((B, Lmax, Hkv, D), 8), _bf16_randn((B, Lmax, Hkv, D), 9)
+    kp = np.concatenate([kc[b, :n] for b, n in enumerate(sl)])
+    vp = np.concatenate([vc[b, :n] for b, n in enumerate(sl)])
+    cu_k = np.concatenate([[0], np.cumsum(sl)])
+    for W, S, full in ((8, 2, False), (1, 0, True)):
+        a = oracle.prefill_chunked(q, kp, vp, np.arange(B + 1), cu_k, W, S, full)
+        b = oracle.decode(q, kc, vc, sl, W, S, full)
+        assert np.array_equal(a["out"], b["out"])
+
+
+def test_packed_batch_sequences_are_independent_and_equal_lengths_reduce_to_prefill():
+    Hq, Hkv, D, W, S = 4, 2, 16, 6, 2
+    lq, lk = [4, 9, 1], [10, 9, 30]
+    qs = [_bf16_randn((n, Hq, D), 10 + i) for i, n in enumerate(lq)]
+    ks = [_bf16_randn((n, Hkv, D), 20 + i) for i, n in enumerate(lk)]
+    vs = [_bf16_randn((n, Hkv, D), 30 + i) for i, n in enumerate(lk)]
+    cq, ck = np.concatenate([[0], np.cumsum(lq)]), np.concatenate([[0], np.cumsum(lk)])
+    packed = oracle.prefill_chunked(np.concatenate(qs), np.concatenate(ks), np.concatenate(vs), cq, ck, W, S, False)
+    for b in range(3):
+        alone = oracle.prefill_chunked(qs[b], ks[b], vs[b], [0, lq[b]], [0, lk[b]], W, S, False)
+        assert np.array_equal(packed["out"][cq[b]:cq[b + 1]], alone["out"])
+    # len_q == len_k everywhere: the self-attention prefill
+    same = oracle.prefill_chunked(np.concatenate(ks).repeat(2, axis=1), np.concatenate(ks), np.concatenate(vs), ck, ck, W, S,
+                                  False)
+    ref = oracle.prefill(np.concatenate(ks).repeat(2, axis=1), np.concatenate(ks), np.concatenate(vs), ck, W, S, False)
+    assert np.array_equal(same["out"], ref["out"])
+
+
+def test_chunked_rejects_more_queries_than_keys():
+    q, k = _bf16_randn((5, 2, 8), 1), _bf16_randn((4, 2, 8), 2)
+    with pytest.raises(ValueError):
+        oracle.prefill_chunked(q, k, k, [0, 5], [0, 4], 4, 0, False)
