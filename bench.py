@@ -346,7 +346,7 @@ def run_ours(args, rank, local_rank, world):
                 "h2d_bytes_per_step": int(q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": int(out.numel()) * 2,
                 "ms_per_step": e2e_ms},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "prefill_kernel<128>", "bound": "tensor", "achieved": achieved,
+        "roofline": {"kernel": "prefill_kernel<128, false>", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                      "traffic": PREFILL_DRAM_TRAFFIC_BYTES, "peak_source": peaks["source"] + " burst bf16",
                      "frac_of_nominal_2250": achieved / 2250.0, "ms_per_launch": avg_pre_ms},

@@ -74,6 +74,25 @@ int swaa_prefill(const void* q, const void* k, const void* v, void* out, const i
                  float* lse, void* stream);
 
 /*
+ * Chunked prefill: the queries of sequence b are the LAST len_q tokens of a context of len_k >= len_q
+ * tokens whose keys and values are all supplied (Sec. 3.1.1 / Fig. 1a: tokens that come later attend to the
+ * stored context under the layer's mask; a serving engine feeds a long prompt in chunks).  Query i of the
+ * chunk sits at position len_k - len_q + i of its sequence; window and n_sink are measured in sequence
+ * positions, not inside the chunk.  With len_q == len_k for every sequence this is swaa_prefill.
+ *
+ *   q, out        device, [Tq, Hq, D] bf16, packed by cu_seqlens_q (int32 [B+1], cu[0] = 0, cu[B] = Tq)
+ *   k, v          device, [Tk, Hkv, D] bf16, packed by cu_seqlens_k (int32 [B+1], cu[0] = 0, cu[B] = Tk)
+ *   max_seqlen_q  upper bound on any len_q (sizes the launch); max_seqlen_k upper bound on any len_k.
+ *   lse           device, float32 [Hq, Tq]; may be NULL.
+ * A sequence with len_q > len_k, or longer than the stated bounds, is reported as SWAA_ERR_BAD_SEQLENS
+ * through the status word and its rows are not written.  Other arguments as for swaa_prefill.
+ */
+int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens_q,
+                         const int32_t* cu_seqlens_k, int B, int Tq, int Tk, int max_seqlen_q, int max_seqlen_k,
+                         int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale, float* lse,
+                         void* stream);
+
+/*
  * Decode: one query token per sequence against a dense KV cache (Sec. 3.1.1 "FA Decode": with is_full
  * the generated token sees the whole context; App. A: the full-context cache is retained).
  *

@@ -23,5 +23,6 @@ from .binding import (  # noqa: F401
     swaa_decode_static,
     DECODE_STATIC_SCRATCH_BYTES,
     swaa_prefill,
+    swaa_prefill_chunked,
     last_device_status,
 )

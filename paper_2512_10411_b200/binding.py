@@ -62,6 +62,8 @@ def load_library():
     vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
     lib.swaa_prefill.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     lib.swaa_prefill.restype = ci
+    lib.swaa_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
+    lib.swaa_prefill_chunked.restype = ci
     lib.swaa_decode_workspace_size.argtypes = [ci] * 8
     lib.swaa_decode_workspace_size.restype = ctypes.c_size_t
     lib.swaa_decode_num_blocks.argtypes = [ci] * 8
@@ -129,6 +131,30 @@ def swaa_prefill(q, k, v, out, cu_seqlens, max_seqlen: int, window: int, n_sink:
                           _dev_ptr(lse, torch.float32, "lse"), _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_prefill")
+
+
+def swaa_prefill_chunked(q, k, v, out, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, window: int,
+                         n_sink: int, is_full: bool, scale: float = 0.0, lse=None, stream=None) -> None:
+    """Forwards to C swaa_prefill_chunked.  q, out [Tq,Hq,D]; k, v [Tk,Hkv,D] bf16; cu_seqlens_* int32 [B+1];
+    lse f32 [Hq,Tq].  The queries of each sequence are the last len_q tokens of its len_k-token context."""
+    lib = load_library()
+    Tq, Hq, D = q.shape
+    Tk, Hkv = k.shape[0], k.shape[1]
+    if tuple(k.shape) != (Tk, Hkv, D) or tuple(v.shape) != (Tk, Hkv, D) or tuple(out.shape) != (Tq, Hq, D):
+        raise ValueError("swaa_prefill_chunked: inconsistent tensor shapes")
+    B = cu_seqlens_q.numel() - 1
+    if cu_seqlens_k.numel() != B + 1:
+        raise ValueError("swaa_prefill_chunked: cu_seqlens_q and cu_seqlens_k must have the same length")
+    if lse is not None and tuple(lse.shape) != (Hq, Tq):
+        raise ValueError("swaa_prefill_chunked: lse must be [Hq, Tq]")
+    bf = torch.bfloat16
+    rc = lib.swaa_prefill_chunked(_dev_ptr(q, bf, "q"), _dev_ptr(k, bf, "k"), _dev_ptr(v, bf, "v"),
+                                  _dev_ptr(out, bf, "out"), _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
+                                  _dev_ptr(cu_seqlens_k, torch.int32, "cu_seqlens_k"), B, Tq, Tk, int(max_seqlen_q),
+                                  int(max_seqlen_k), Hq, Hkv, D, int(window), int(n_sink), int(bool(is_full)),
+                                  float(scale), _dev_ptr(lse, torch.float32, "lse"), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_prefill_chunked")
 
 
 def decode_workspace_size(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) -> int:

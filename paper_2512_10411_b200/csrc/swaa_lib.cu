@@ -227,59 +227,69 @@ static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H
     return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
-template <int D>
+template <int D, bool kChunked>
 static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                           const PrefillParams& p, int sm_count, cudaStream_t st) {
     using L = PrefillSmem<D>;
-    if (cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(prefill_kernel<D, kChunked>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             L::kDynamicBytes) != cudaSuccess)
         return SWAA_ERR_CUDA;
     // persistent blocks: one per SM (or fewer when there is less work), each walks its share of the items
     long long blocks = (long long)p.n_pairs * p.tiles_ub;
     if (blocks > sm_count) blocks = sm_count;
-    prefill_kernel<D><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, p);
+    prefill_kernel<D, kChunked><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
 }  // namespace swaa
 
-extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens, int B,
-                            int T, int max_seqlen, int Hq, int Hkv, int D, int window, int n_sink, int is_full,
-                            float scale, float* lse, void* stream) {
-    if (B < 0 || T < 0 || max_seqlen < 0 || Hq < 1 || Hkv < 1 || n_sink < 0) return SWAA_ERR_INVALID_ARG;
+namespace swaa {
+
+// Shared body of swaa_prefill (cu_seqlens_k == nullptr: keys are packed like the queries) and
+// swaa_prefill_chunked.
+static int prefill_impl(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens_q,
+                        const int32_t* cu_seqlens_k, int B, int Tq, int Tk, int max_seqlen_q, int max_seqlen_k, int Hq,
+                        int Hkv, int D, int window, int n_sink, int is_full, float scale, float* lse, void* stream) {
+    if (B < 0 || Tq < 0 || Tk < 0 || max_seqlen_q < 0 || max_seqlen_k < 0 || Hq < 1 || Hkv < 1 || n_sink < 0)
+        return SWAA_ERR_INVALID_ARG;
     if (!is_full && window < 1) return SWAA_ERR_INVALID_ARG;
     if (Hq % Hkv != 0 || (D != 64 && D != 128)) return SWAA_ERR_UNSUPPORTED;
-    if (B == 0 || T == 0) return SWAA_OK;
-    if (!q || !k || !v || !out || !cu_seqlens) return SWAA_ERR_INVALID_ARG;
+    if (B == 0 || Tq == 0) return SWAA_OK;
+    if (!q || !k || !v || !out || !cu_seqlens_q) return SWAA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(cu_seqlens) & 3u) != 0 || (reinterpret_cast<uintptr_t>(lse) & 3u) != 0)
+    if ((reinterpret_cast<uintptr_t>(cu_seqlens_q) & 3u) != 0 || (reinterpret_cast<uintptr_t>(cu_seqlens_k) & 3u) != 0 ||
+        (reinterpret_cast<uintptr_t>(lse) & 3u) != 0)
         return SWAA_ERR_INVALID_ARG;
+    if (Tk < Tq) return SWAA_ERR_INVALID_ARG;
     DeviceInfo info;
     int rc = current_device_info(&info);
     if (rc != SWAA_OK) return rc;
     if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
 
     CUtensorMap tq, tk, tv, to;
-    if ((rc = make_token_major_map(&tq, q, T, Hq, D)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&tk, k, T, Hkv, D)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&tv, v, T, Hkv, D)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&to, out, T, Hq, D, 32)) != SWAA_OK) return rc;  // output rows, 32 at a time
+    if ((rc = make_token_major_map(&tq, q, Tq, Hq, D)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tk, k, Tk, Hkv, D)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tv, v, Tk, Hkv, D)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&to, out, Tq, Hq, D, 32)) != SWAA_OK) return rc;  // output rows, 32 at a time
 
     PrefillParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lse = lse;
-    p.cu_seqlens = cu_seqlens;
+    p.cu_seqlens = cu_seqlens_q;
+    p.cu_seqlens_k = cu_seqlens_k;
     p.B = B;
-    p.T = T;
-    p.max_seqlen = max_seqlen;
+    p.T = Tq;
+    p.Tk = Tk;
+    p.max_seqlen = max_seqlen_q;
+    p.max_seqlen_k = max_seqlen_k;
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.G = Hq / Hkv;
     p.pairs_per_kv = (p.G + 1) / 2;
     p.n_pairs = Hkv * p.pairs_per_kv;
-    const long long ub_a = (long long)T / kPrefillBM + B;
-    const long long ub_b = (long long)B * ((max_seqlen + kPrefillBM - 1) / kPrefillBM);
+    const long long ub_a = (long long)Tq / kPrefillBM + B;
+    const long long ub_b = (long long)B * ((max_seqlen_q + kPrefillBM - 1) / kPrefillBM);
     const long long ub = ub_a < ub_b ? ub_a : ub_b;
     if (ub > 2147483647LL / p.n_pairs) return SWAA_ERR_UNSUPPORTED;
     p.tiles_ub = (int)ub;
@@ -290,8 +300,29 @@ extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* o
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
     p.sl2 = p.scale * 1.4426950408889634f;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return D == 128 ? launch_prefill<128>(tq, tk, tv, to, p, info.sm_count, st)
-                    : launch_prefill<64>(tq, tk, tv, to, p, info.sm_count, st);
+    if (cu_seqlens_k != nullptr)
+        return D == 128 ? launch_prefill<128, true>(tq, tk, tv, to, p, info.sm_count, st)
+                        : launch_prefill<64, true>(tq, tk, tv, to, p, info.sm_count, st);
+    return D == 128 ? launch_prefill<128, false>(tq, tk, tv, to, p, info.sm_count, st)
+                    : launch_prefill<64, false>(tq, tk, tv, to, p, info.sm_count, st);
+}
+
+}  // namespace swaa
+
+extern "C" int swaa_prefill(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens, int B,
+                            int T, int max_seqlen, int Hq, int Hkv, int D, int window, int n_sink, int is_full,
+                            float scale, float* lse, void* stream) {
+    return prefill_impl(q, k, v, out, cu_seqlens, nullptr, B, T, T, max_seqlen, max_seqlen, Hq, Hkv, D, window, n_sink,
+                        is_full, scale, lse, stream);
+}
+
+extern "C" int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out,
+                                    const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k, int B, int Tq, int Tk,
+                                    int max_seqlen_q, int max_seqlen_k, int Hq, int Hkv, int D, int window, int n_sink,
+                                    int is_full, float scale, float* lse, void* stream) {
+    if (!cu_seqlens_k) return SWAA_ERR_INVALID_ARG;
+    return prefill_impl(q, k, v, out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq, Hkv, D,
+                        window, n_sink, is_full, scale, lse, stream);
 }
 
 // ------------------------------------------------------------------- decode without allocation

@@ -40,8 +40,10 @@ constexpr float kRescaleThreshold = 8.0f;                   // log2 units
 struct PrefillParams {
     __nv_bfloat16* out;
     float* lse;             // nullable, [Hq, T]
-    const int32_t* cu_seqlens;
+    const int32_t* cu_seqlens;    // queries (and keys, when cu_seqlens_k is null)
+    const int32_t* cu_seqlens_k;  // nullable: keys of a chunked prefill, len_k >= len_q per sequence
     int B, T, max_seqlen, Hq, Hkv, G;
+    int Tk, max_seqlen_k;         // packed key tokens and longest key sequence (chunked prefill only)
     int pairs_per_kv;       // ceil(G / 2)
     int n_pairs;            // Hkv * pairs_per_kv
     int tiles_ub;           // upper bound on the number of query tiles over all sequences
@@ -233,9 +235,13 @@ struct PrefillSmem {
 // One unit of work: a 128-row query tile of one sequence for one pair of query heads.
 struct WorkItem {
     int valid, seq_start, seq_len, m_tile, pair;
+    int k_start;  // first packed key token of the sequence (= seq_start for self attention)
+    int k_off;    // position of the sequence's first query inside its sequence: len_k - len_q (0 for self attention)
 };
 
-template <int D>
+// kChunked: queries are the last len_q tokens of a longer key sequence (separate packing of the keys).
+// The self-attention instance compiles the offsets away.
+template <int D, bool kChunked>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -296,6 +302,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         w.seq_len = d[2];
         w.m_tile = d[3];
         w.pair = d[4];
+        w.k_start = kChunked ? d[5] : w.seq_start;
+        w.k_off = kChunked ? d[6] : 0;
         if (release) mbar_arrive(bar(BAR_WE + slot));
         return true;
     };
@@ -309,7 +317,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // descriptors.  Items are ordered heavy-first: last sequence first, last tile of a sequence first.
         if (lane == 0) {
             if (p.cu_seqlens[0] != 0 || p.cu_seqlens[p.B] != p.T) record_device_error(SWAA_ERR_BAD_SEQLENS);
-            int b = p.B, acc = 0, cur_nt = 0, cur_s = 0, cur_len = 0;
+            int b = p.B, acc = 0, cur_nt = 0, cur_s = 0, cur_len = 0, cur_ks = 0, cur_off = 0;
             auto next_seq = [&]() {
                 acc += cur_nt;
                 --b;
@@ -320,6 +328,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (len < 0 || len > p.max_seqlen || s0 < 0 || e0 > p.T) {
                         record_device_error(SWAA_ERR_BAD_SEQLENS);
                         len = 0;
+                    }
+                    cur_ks = s0;
+                    cur_off = 0;
+                    if (kChunked) {  // chunked prefill: the queries are the last `len` tokens
+                        const int ks = p.cu_seqlens_k[b], ke = p.cu_seqlens_k[b + 1];
+                        if (ke - ks < len || ke - ks > p.max_seqlen_k || ks < 0 || ke > p.Tk) {
+                            record_device_error(SWAA_ERR_BAD_SEQLENS);
+                            len = 0;
+                        }
+                        cur_ks = ks;
+                        cur_off = ke - ks - len;
                     }
                     cur_s = s0;
                     cur_len = len;
@@ -340,6 +359,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 d[2] = cur_len;
                 d[3] = b >= 0 ? cur_nt - 1 - (int)(tile_id - acc) : 0;
                 d[4] = pair;
+                if (kChunked) {
+                    d[5] = cur_ks;
+                    d[6] = cur_off;
+                }
                 mbar_arrive(bar(BAR_WF + slot));
                 if (b < 0) break;
             }
@@ -359,7 +382,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
                 const bool hasB = (hA + 1) < (hk + 1) * p.G;
                 const int i0 = w.m_tile * BM, i1 = min(w.seq_len, i0 + BM) - 1;
-                const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
+                const TileRange tr = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, p.n_sink, full);
                 const int nt = tr.count();
                 // Q tiles of both sides (the previous item's last QK must have retired)
                 ok = mbar_wait(bar(BAR_QE), ((uint32_t)items & 1u) ^ 1u, abort_flag);
@@ -377,7 +400,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 for (int n = 0; n < nt; ++n, ++g) {
                     const int s = g % ST;
                     const uint32_t ph = (uint32_t)(g / ST) & 1u;
-                    const int tk = w.seq_start + tr.tile(n) * BN;
+                    const int tk = w.k_start + tr.tile(n) * BN;
                     ok = mbar_wait(bar(BAR_KE + s), ph ^ 1u, abort_flag);
                     if (!ok) break;
                     mbar_arrive_expect_tx(bar(BAR_KF + s), (uint32_t)L::kTileBytes);
@@ -462,7 +485,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
                 const bool hasB = (hA + 1) < (hk + 1) * p.G;
                 const int i0 = w.m_tile * BM, i1 = min(w.seq_len, i0 + BM) - 1;
-                const int nt = tile_range(i0, i1, BN, p.window, p.n_sink, full).count();
+                const int nt = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, p.n_sink, full).count();
                 ok = mbar_wait(bar(BAR_QF), (uint32_t)items & 1u, abort_flag) &&
                      mbar_wait(bar(BAR_KF + g % ST), (uint32_t)(g / ST) & 1u, abort_flag);
                 if (!ok) break;
@@ -550,10 +573,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const bool hasB = (hA + 1) < (hk + 1) * p.G;
             if (side == 1 && !hasB) continue;
             const int seq_start = w.seq_start, seq_len = w.seq_len;
-            const int i0 = w.m_tile * BM, i1 = min(seq_len, i0 + BM) - 1;
+            const int q0 = w.m_tile * BM;    // first query of the tile, counted inside the sequence's queries
+            const int iq = q0 + row;         // this thread's query, same counting
+            const int i0 = q0 + w.k_off, i1 = min(seq_len, q0 + BM) - 1 + w.k_off;  // positions inside the sequence
             const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
             const int nt = tr.count();
-            const int i = i0 + row;  // position of this thread's query inside its sequence
+            const int i = iq + w.k_off;      // position of this thread's query inside its sequence
             const int h = hA + side;
             float m_used = -INFINITY, l_sum = 0.f;
             for (int n = 0; n < nt; ++n, ++gs) {
@@ -691,7 +716,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mbar_arrive(bar(BAR_OF + side));  // O may be overwritten by the next item's first PV
             SWAA_TICK(e1);
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            if (i0 + wq * 32 + 31 < seq_len) {
+            if (q0 + wq * 32 + 31 < seq_len) {
                 // all 32 rows of this warp are valid: stage [32 rows][64 ch] panels in shared memory in the
                 // 128-byte-swizzled layout and let TMA write them (fully coalesced, off the LSU path)
                 const uint32_t stage = sStage + (uint32_t)warp * 4096u;
@@ -711,13 +736,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_3d(&tm_o, stage, pn * 64, h, seq_start + i0 + wq * 32);
+                        tma_store_3d(&tm_o, stage, pn * 64, h, seq_start + q0 + wq * 32);
                         tma_store_commit();
                     }
                 }
-            } else if (i < seq_len) {
+            } else if (iq < seq_len) {
                 // ragged tail of a sequence: plain predicated row stores
-                __nv_bfloat16* orow = p.out + ((size_t)(seq_start + i) * p.Hq + h) * D;
+                __nv_bfloat16* orow = p.out + ((size_t)(seq_start + iq) * p.Hq + h) * D;
 #pragma unroll
                 for (int v = 0; v < D / 8; ++v) {
                     uint4 o4;
@@ -728,9 +753,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     *reinterpret_cast<uint4*>(orow + v * 8) = o4;
                 }
             }
-            if (i < seq_len && p.lse != nullptr) {
+            if (iq < seq_len && p.lse != nullptr) {
                 const float lse2 = (m_used == -INFINITY) ? -INFINITY : m_used * p.sl2 + log2f(l_sum);
-                p.lse[(size_t)h * p.T + seq_start + i] = lse2 * 0.6931471805599453f;
+                p.lse[(size_t)h * p.T + seq_start + iq] = lse2 * 0.6931471805599453f;
             }
 #ifdef SWAA_PHASE_TIMING
             if (lane == 0 && wq == 0) {
