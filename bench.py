@@ -452,6 +452,77 @@ def run_sweep():
     time_case("cfg2_full_causal", inputs.cfg_long(is_full=True), True, reps=3)
     time_case("cfg5_varlen", inputs.cfg_varlen(), False, reps=3)
     time_case("cfg1_tiny", inputs.cfg_tiny(), False)
+    # chunked prefill: a 4096-token chunk at the end of a 131072-token context (heads and mask of workload 2)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    lq, lk, Hq, Hkv, D, W, S = 4096, 131072, 32, 8, 128, 2048, 4
+    cq = torch.randn((lq, Hq, D), generator=g, device="cuda").to(torch.bfloat16)
+    ck = torch.randn((lk, Hkv, D), generator=g, device="cuda").to(torch.bfloat16)
+    cv = torch.randn((lk, Hkv, D), generator=g, device="cuda").to(torch.bfloat16)
+    cuq = torch.tensor([0, lq], dtype=torch.int32, device="cuda")
+    cuk = torch.tensor([0, lk], dtype=torch.int32, device="cuda")
+    cout = torch.empty_like(cq)
+    for full in (False, True):
+        ms = []
+        for r in range(6):
+            flush.zero_()
+            flush_rd.sum()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            swaa.swaa_prefill_chunked(cq, ck, cv, cout, cuq, cuk, lq, lk, W, S, full)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if r > 0:
+                ms.append(a.elapsed_time(b))
+        assert swaa.last_device_status() == 0
+        ms.sort()
+        pairs = sum(lk - lq + i + 1 for i in range(lq)) if full else lq * (W + S)
+        tf = 4.0 * D * Hq * pairs / (ms[len(ms) // 2] * 1e-3) / 1e12
+        print(json.dumps({"case": "chunked_prefill", "len_q": lq, "len_k": lk, "Hq": Hq, "Hkv": Hkv, "D": D, "window": W,
+                          "n_sink": S, "is_full": full, "ms": ms[len(ms) // 2], "effective_tflops": tf,
+                          "frac_of_measured_peak": tf / peaks["bf16_tflops"]}), flush=True)
+    del cq, ck, cv, cout
+    # paged decode: workload 4 with 256-entry pages handed out in random order, against the dense layout
+    dcfg = inputs.cfg_decode()
+    dq, kc, vc, sl = inputs.make_decode_inputs(dcfg, "cuda")
+    page = 256
+    nblk = dcfg.Lmax // page
+    perm = torch.randperm(dcfg.B * nblk, generator=g, device="cuda")
+    bt = perm.view(dcfg.B, nblk).to(torch.int32).contiguous()
+    kp = torch.empty((dcfg.B * nblk, page, dcfg.Hkv, dcfg.D), dtype=torch.bfloat16, device="cuda")
+    vp = torch.empty_like(kp)
+    kp[perm] = kc.view(dcfg.B * nblk, page, dcfg.Hkv, dcfg.D)
+    vp[perm] = vc.view(dcfg.B * nblk, page, dcfg.Hkv, dcfg.D)
+    dout = torch.empty_like(dq)
+    for full in (True, False):
+        nbytes = float(dcfg.B) * (dcfg.Lmax if full else dcfg.window + dcfg.n_sink) * dcfg.Hkv * dcfg.D * 4
+        ws_d = torch.empty(swaa.decode_workspace_size(dcfg.B, dcfg.Hq, dcfg.Hkv, dcfg.D, dcfg.Lmax, dcfg.window,
+                                                      dcfg.n_sink, full), dtype=torch.uint8, device="cuda")
+        ws_p = torch.empty(swaa.decode_paged_workspace_size(dcfg.B, dcfg.Hq, dcfg.Hkv, dcfg.D, nblk, page, dcfg.window,
+                                                            dcfg.n_sink, full), dtype=torch.uint8, device="cuda")
+        res = {}
+        for kind in ("dense", "paged"):
+            us = []
+            for r in range(11):
+                flush.zero_()
+                flush_rd.sum()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                if kind == "dense":
+                    swaa.swaa_decode(dq, kc, vc, dout, sl, dcfg.window, dcfg.n_sink, full, ws_d)
+                else:
+                    swaa.swaa_decode_paged(dq, kp, vp, dout, bt, sl, dcfg.window, dcfg.n_sink, full, ws_p)
+                b.record(stream)
+                torch.cuda.synchronize()
+                if r > 0:
+                    us.append(1e3 * a.elapsed_time(b))
+            us.sort()
+            res[kind] = us[len(us) // 2]
+        assert swaa.last_device_status() == 0
+        print(json.dumps({"case": "decode_paged_vs_dense", "is_full": full, "page_size": page, "bytes": nbytes,
+                          "dense_us": res["dense"], "dense_gbs": nbytes / res["dense"] / 1e3,
+                          "paged_us": res["paged"], "paged_gbs": nbytes / res["paged"] / 1e3,
+                          "hbm_peak_gbs": peaks["hbm_gbs"]}), flush=True)
+    del kc, vc, kp, vp
     # workload 3: the 36-layer interleaved stack, per layer and in total (mask policy from the layer schedule)
     pol = swaa.SwaaPolicy(n_layers=36, window=4096, n_sink=64, fa_start=3, fa_step=4, fa_decode=True)
     total, per_kind = 0.0, {False: [], True: []}

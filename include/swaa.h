@@ -118,6 +118,27 @@ int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out
                 size_t workspace_bytes, void* stream);
 
 /*
+ * Decode against a paged KV cache (the layout of serving engines such as the vLLM integration of Sec. 4.1.1:
+ * the cache of a sequence is a list of fixed-size pages anywhere in a common pool).
+ *
+ *   kpages, vpages  device, [num_pages, page_size, Hkv, D] bf16; page_size is a multiple of 64.
+ *   block_table     device, int32 [B, max_blocks]; entry j of sequence b lives in page
+ *                   block_table[b][j / page_size] at row j % page_size.  Only the entries that cover
+ *                   seqlens[b] are read.  A page index outside [0, num_pages) is reported as
+ *                   SWAA_ERR_BAD_SEQLENS through the status word (the page then reads as zeros).
+ *   seqlens         device, int32 [B]; 1 <= seqlens[b] <= max_blocks * page_size, as for swaa_decode.
+ *   workspace       at least swaa_decode_paged_workspace_size(...) bytes, 256-byte aligned, uninitialised.
+ * Same computation, mask policy, status codes and in-launch combine as swaa_decode.
+ */
+size_t swaa_decode_paged_workspace_size(int B, int Hq, int Hkv, int D, int max_blocks, int page_size, int window,
+                                        int n_sink, int is_full);
+
+int swaa_decode_paged(const void* q, const void* kpages, const void* vpages, void* out, const int32_t* block_table,
+                      const int32_t* seqlens, int B, int max_blocks, int num_pages, int page_size, int Hq, int Hkv,
+                      int D, int window, int n_sink, int is_full, float scale, void* workspace, size_t workspace_bytes,
+                      void* stream);
+
+/*
  * Allocation-free decode.  (The paper has no counterpart to this call; it exists for integration.)
  *
  * Same computation and arguments as swaa_decode, but the split-K scratch lives in a fixed array inside

@@ -9,6 +9,7 @@ from .swaa_oracle import (  # noqa: F401
     build,
     count_pairs,
     decode,
+    decode_paged,
     layer_is_full,
     num_threads,
     prefill,

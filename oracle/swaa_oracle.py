@@ -179,3 +179,22 @@ def decode(q, kcache, vcache, seqlens, window: int, n_sink: int, is_full: bool, 
     if rc != 0:
         raise ValueError("swaa_oracle_decode: inconsistent arguments")
     return {"out": out, "lse": lse, "psum": psum, "nvis": nvis}
+
+
+def decode_paged(q, kpages, vpages, block_table, seqlens, window: int, n_sink: int, is_full: bool,
+                 scale: float | None = None):
+    """Decode against a paged cache, by definition: entry j of sequence b is row j % page_size of page
+    block_table[b][j // page_size]; the entries are gathered into a dense cache (pure indexing) and handed
+    to the dense decode.  kpages, vpages [num_pages, page_size, Hkv, D]; block_table [B, max_blocks]."""
+    kpages, vpages = _f32(kpages), _f32(vpages)
+    bt = np.asarray(block_table, dtype=np.int64)
+    sl = np.asarray(seqlens, dtype=np.int64)
+    B, page_size = bt.shape[0], kpages.shape[1]
+    Lmax = int(sl.max())
+    kd = np.zeros((B, Lmax) + kpages.shape[2:], dtype=np.float32)
+    vd = np.zeros_like(kd)
+    for b in range(B):
+        j = np.arange(int(sl[b]))
+        kd[b, j] = kpages[bt[b, j // page_size], j % page_size]
+        vd[b, j] = vpages[bt[b, j // page_size], j % page_size]
+    return decode(q, kd, vd, sl, window, n_sink, is_full, scale)

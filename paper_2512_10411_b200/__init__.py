@@ -20,6 +20,8 @@ from .binding import (  # noqa: F401
     schedule_is_full,
     status_str,
     swaa_decode,
+    swaa_decode_paged,
+    decode_paged_workspace_size,
     swaa_decode_static,
     DECODE_STATIC_SCRATCH_BYTES,
     swaa_prefill,

@@ -70,6 +70,10 @@ def load_library():
     lib.swaa_decode_num_blocks.restype = ci
     lib.swaa_decode.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
     lib.swaa_decode.restype = ci
+    lib.swaa_decode_paged_workspace_size.argtypes = [ci] * 9
+    lib.swaa_decode_paged_workspace_size.restype = ctypes.c_size_t
+    lib.swaa_decode_paged.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
+    lib.swaa_decode_paged.restype = ci
     lib.swaa_decode_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp]
     lib.swaa_decode_static.restype = ci
     lib.swaa_schedule_is_full.argtypes = [ctypes.POINTER(_Policy), ci, ci]
@@ -185,6 +189,33 @@ def swaa_decode(q, kcache, vcache, out, seqlens, window: int, n_sink: int, is_fu
                          _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_decode")
+
+
+def decode_paged_workspace_size(B, Hq, Hkv, D, max_blocks, page_size, window, n_sink, is_full) -> int:
+    """Forwards to C swaa_decode_paged_workspace_size (bytes)."""
+    return int(load_library().swaa_decode_paged_workspace_size(B, Hq, Hkv, D, int(max_blocks), int(page_size),
+                                                               int(window), int(n_sink), int(bool(is_full))))
+
+
+def swaa_decode_paged(q, kpages, vpages, out, block_table, seqlens, window: int, n_sink: int, is_full: bool, workspace,
+                      scale: float = 0.0, stream=None) -> None:
+    """Forwards to C swaa_decode_paged.  q, out [B,Hq,D]; kpages, vpages [num_pages,page_size,Hkv,D] bf16;
+    block_table int32 [B,max_blocks]; seqlens int32 [B]; workspace uint8 of decode_paged_workspace_size(...) bytes."""
+    lib = load_library()
+    B, Hq, D = q.shape
+    num_pages, page_size, Hkv, _ = kpages.shape
+    if tuple(vpages.shape) != tuple(kpages.shape) or kpages.shape[3] != D or tuple(out.shape) != (B, Hq, D):
+        raise ValueError("swaa_decode_paged: inconsistent tensor shapes")
+    if block_table.dim() != 2 or block_table.shape[0] != B or seqlens.numel() != B:
+        raise ValueError("swaa_decode_paged: block_table must be [B, max_blocks] and seqlens [B]")
+    bf = torch.bfloat16
+    rc = lib.swaa_decode_paged(_dev_ptr(q, bf, "q"), _dev_ptr(kpages, bf, "kpages"), _dev_ptr(vpages, bf, "vpages"),
+                               _dev_ptr(out, bf, "out"), _dev_ptr(block_table, torch.int32, "block_table"),
+                               _dev_ptr(seqlens, torch.int32, "seqlens"), B, block_table.shape[1], num_pages, page_size,
+                               Hq, Hkv, D, int(window), int(n_sink), int(bool(is_full)), float(scale),
+                               _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_decode_paged")
 
 
 DECODE_STATIC_SCRATCH_BYTES = 2 << 20

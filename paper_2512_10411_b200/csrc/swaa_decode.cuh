@@ -46,6 +46,9 @@ struct DecodeParams {
     unsigned long long* tickets;  // [gridDim.x]; (call stamp << 16 | arrivals), needs no initialisation
     unsigned long long stamp;     // 48-bit number unique to this call (never 0)
     float* part;   // [2 * gridDim.x][8*NH][D + 2]: per head (max in score units, sum, unnormalised O)
+    // paged cache only: entry j of sequence b lives in page block_table[b * max_blocks + j / page_size]
+    const int32_t* block_table;
+    int max_blocks, page_tiles /* page_size / 64 */, num_pages;
 };
 
 constexpr int kDecodeTileKeys = 64;
@@ -79,29 +82,35 @@ struct SeqGeom {
     int ns;   // sink keys that lie before the window
     int nst;  // sink tiles
     int nt;   // tiles per item
+    int w0;   // first key of the first window tile: lo (dense cache), or lo rounded down to a tile (paged cache)
 };
 
-__host__ __device__ inline SeqGeom decode_seq_geom(int len, int Lmax, int window, int n_sink, int is_full) {
+// With `aligned` the window tiles start on multiples of the tile size, so that no tile straddles a page of
+// a paged cache; the keys before `lo` in the first window tile are then masked like those past `len`.
+__host__ __device__ inline SeqGeom decode_seq_geom(int len, int Lmax, int window, int n_sink, int is_full,
+                                                   bool aligned = false) {
     SeqGeom s;
     if (len < 1 || len > Lmax) {
-        s.len = s.lo = s.ns = s.nst = s.nt = 0;
+        s.len = s.lo = s.ns = s.nst = s.nt = s.w0 = 0;
         return s;
     }
     s.len = len;
     s.lo = is_full ? 0 : (len > window ? len - window : 0);
     s.ns = is_full ? 0 : (n_sink < s.lo ? n_sink : s.lo);
     s.nst = (s.ns + kDecodeTileKeys - 1) / kDecodeTileKeys;
-    s.nt = s.nst + (len - s.lo + kDecodeTileKeys - 1) / kDecodeTileKeys;
+    s.w0 = aligned ? s.lo / kDecodeTileKeys * kDecodeTileKeys : s.lo;
+    s.nt = s.nst + (len - s.w0 + kDecodeTileKeys - 1) / kDecodeTileKeys;
     return s;
 }
 
 // Position in the global tile list; every role of a block walks the same positions.
+template <bool kPaged>
 struct DecodeWalker {
     int b, hv, ti;
     SeqGeom s;
     __device__ __forceinline__ void seek(const DecodeParams& p, int b0, long long off) {
         b = b0;
-        s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
+        s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full, kPaged);
         hv = (int)(off / s.nt);
         ti = (int)(off - (long long)hv * s.nt);
     }
@@ -111,16 +120,18 @@ struct DecodeWalker {
         if (++hv < p.IPB) return;
         hv = 0;
         while (++b < p.B) {
-            s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full);
+            s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full, kPaged);
             if (s.nt > 0) return;
         }
         s.nt = 0;  // past the last sequence
     }
-    __device__ __forceinline__ int key0() const { return ti < s.nst ? ti * kDecodeTileKeys : s.lo + (ti - s.nst) * kDecodeTileKeys; }
-    __device__ __forceinline__ int valid() const {  // visible keys in this tile, 1 .. 64
+    __device__ __forceinline__ int key0() const { return ti < s.nst ? ti * kDecodeTileKeys : s.w0 + (ti - s.nst) * kDecodeTileKeys; }
+    // rows [vbegin, vend) of this tile hold visible keys; vbegin > 0 only in the first window tile of a paged cache
+    __device__ __forceinline__ int vend() const {
         const int left = ti < s.nst ? s.ns - ti * kDecodeTileKeys : s.len - key0();
         return left < kDecodeTileKeys ? left : kDecodeTileKeys;
     }
+    __device__ __forceinline__ int vbegin() const { return (kPaged && ti == s.nst) ? s.lo - s.w0 : 0; }
 };
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -149,7 +160,7 @@ __device__ unsigned long long g_decode_stamps[256][8];
 #define SWAA_DSTAMP(slot)
 #endif
 
-template <int D, int NH>
+template <int D, int NH, bool kPaged>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
               const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16, const DecodeParams p) {
@@ -199,7 +210,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 
     // ---- where does this block's run of the global tile list start?  (scan of tiles per sequence)
     auto tiles_of = [&](int b) -> long long {
-        return (long long)decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full).nt * p.IPB;
+        return (long long)decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full, kPaged).nt * p.IPB;
     };
     auto zero_fill_bad = [&](int b) {  // a sequence without tiles: report it, zero its output rows (one block does)
         record_device_error(SWAA_ERR_BAD_SEQLENS);
@@ -296,7 +307,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     if (warp == kDecodeConsumerWarps) {
         // =========================================================================== TMA producer
         if (lane == 0) {
-            DecodeWalker w;
+            DecodeWalker<kPaged> w;
             w.seek(p, b0, off0);
             bool ok = true;
             int n = 0, s = 0;
@@ -305,20 +316,30 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 ok = mbar_wait(bar_e(s), ph ^ 1u, abort_flag);
                 if (!ok) break;
                 const int key0 = w.key0(), hk = w.hv / p.HG;
+                int c2 = key0, c3 = w.b;  // TMA coordinates: (entry, sequence) or (row in page, page)
+                if (kPaged) {
+                    const int tile = key0 / kDecodeTileKeys;
+                    c3 = __ldg(p.block_table + (size_t)w.b * p.max_blocks + tile / p.page_tiles);
+                    c2 = (tile % p.page_tiles) * kDecodeTileKeys;
+                    if (c3 < 0 || c3 >= p.num_pages) {
+                        record_device_error(SWAA_ERR_BAD_SEQLENS);
+                        c3 = p.num_pages;  // out of range: the copy delivers zeros
+                    }
+                }
                 const uint32_t dst = smem_base + (uint32_t)s * L::kStageBytes;
                 // a tile with at most 16 visible keys (typically the sinks) is fetched with the 16-row box
-                const bool small = w.valid() <= kDecodeSmallBoxKeys;
+                const bool small = w.vend() <= kDecodeSmallBoxKeys;
                 const CUtensorMap* mk = small ? &tm_k16 : &tm_k;
                 const CUtensorMap* mv = small ? &tm_v16 : &tm_v;
                 const uint32_t bytes = small ? (uint32_t)(L::kPanels * kDecodeSmallBoxKeys * 128) : (uint32_t)L::kTileBytes;
                 mbar_arrive_expect_tx(bar_kf(s), bytes);
 #pragma unroll
                 for (int pn = 0; pn < L::kPanels; ++pn)
-                    tma_load_4d(dst + pn * L::kPanelBytes, mk, pn * 64, hk, key0, w.b, bar_kf(s));
+                    tma_load_4d(dst + pn * L::kPanelBytes, mk, pn * 64, hk, c2, c3, bar_kf(s));
                 mbar_arrive_expect_tx(bar_vf(s), bytes);
 #pragma unroll
                 for (int pn = 0; pn < L::kPanels; ++pn)
-                    tma_load_4d(dst + L::kTileBytes + pn * L::kPanelBytes, mv, pn * 64, hk, key0, w.b, bar_vf(s));
+                    tma_load_4d(dst + L::kTileBytes + pn * L::kPanelBytes, mv, pn * 64, hk, c2, c3, bar_vf(s));
                 if (++s == ST) {
                     s = 0;
                     ph ^= 1u;
@@ -348,7 +369,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const int vrow = 16 * warp + (lane & 7) + 8 * (lane >> 4);        // V: matrices (channels lo/hi) x (keys lo/hi)
     const int vchk = (lane >> 3) & 1;
 
-    DecodeWalker w;
+    DecodeWalker<kPaged> w;
     w.seek(p, b0, off0);
     bool ok = true;
     bool first_seg = true;
@@ -387,11 +408,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
 
         for (int j = 0; j < seg_tiles; ++j, ++n, w.next(p)) {
-            const int vw = w.valid() - 16 * warp;  // visible keys among this warp's 16
+            const int vw = w.vend() - 16 * warp;            // this warp's keys [vb, vw) of its 16 are visible
+            const int vb = kPaged ? max(w.vbegin() - 16 * warp, 0) : 0;
             const uint32_t stage = smem_base + (uint32_t)s * L::kStageBytes;
             ok = ok && mbar_wait(bar_kf(s), ph, abort_flag);
             if (warp == 0 && n == 0) SWAA_DSTAMP(2);  // first K tile landed
-            if (ok && vw > 0) {
+            if (ok && min(vw, 16) > vb) {  // some of this warp's 16 keys are visible
                 // ---- S^T = K Q^T : rows = keys (g, g+8), cols = heads (2c, 2c+1)
                 float sacc[NH][4];
 #pragma unroll
@@ -408,7 +430,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
 
                 // ---- online softmax over this warp's 16 keys
-                const bool ok0 = g < vw, ok1 = g + 8 < vw;
+                const bool ok0 = g < vw && g >= vb, ok1 = g + 8 < vw && g + 8 >= vb;
                 uint32_t pb[NH][2];
 #pragma unroll
                 for (int nh = 0; nh < NH; ++nh) {
@@ -421,7 +443,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
                         bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
                         bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
-                        const float m_new = fmaxf(m_run[nh][e], bm);  // finite: the warp's first key is visible
+                        const float m_new = fmaxf(m_run[nh][e], bm);  // finite: one of the warp's keys is visible
                         alpha[e] = ex2f((m_run[nh][e] - m_new) * p.sl2);
                         m_run[nh][e] = m_new;
                         const float off = m_new * p.sl2;
@@ -449,8 +471,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 ok = mbar_wait(bar_vf(s), ph, abort_flag);
                 if (ok) {
                     // rows of the tile past the last visible key may hold anything (also NaN): clear them
-                    const uint32_t mlo = (2 * c < vw ? 0x0000ffffu : 0u) | (2 * c + 1 < vw ? 0xffff0000u : 0u);
-                    const uint32_t mhi = (2 * c + 8 < vw ? 0x0000ffffu : 0u) | (2 * c + 9 < vw ? 0xffff0000u : 0u);
+                    auto vis = [&](int key) { return key < vw && key >= vb; };
+                    const uint32_t mlo = (vis(2 * c) ? 0x0000ffffu : 0u) | (vis(2 * c + 1) ? 0xffff0000u : 0u);
+                    const uint32_t mhi = (vis(2 * c + 8) ? 0x0000ffffu : 0u) | (vis(2 * c + 9) ? 0xffff0000u : 0u);
 #pragma unroll
                     for (int qb = 0; qb < NKK; ++qb) {
                         const int chunk16 = 2 * qb + vchk;
@@ -458,7 +481,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         ldmatrix_x4_trans(stage + (uint32_t)(L::kTileBytes + (chunk16 >> 3) * L::kPanelBytes + vrow * 128 +
                                                              (((chunk16 & 7) ^ (vrow & 7)) << 4)),
                                           a0, a1, a2, a3);
-                        if (vw < 16) {
+                        if (vw < 16 || vb > 0) {
                             a0 &= mlo;
                             a1 &= mlo;
                             a2 &= mhi;

@@ -54,13 +54,13 @@ struct DecodePlan {
 // One block per SM, fewer when the whole problem has fewer tiles than that.  Depends only on the
 // shape arguments and the SM count (sequence lengths are read on the device).
 static DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full,
-                              int sm_count) {
+                              int sm_count, bool paged = false) {
     DecodePlan pl;
     const int G = Hq / Hkv;
     pl.NH = G > 8 ? 2 : 1;
     const int HC = 8 * pl.NH;
     pl.HG = (G + HC - 1) / HC;
-    const SeqGeom longest = decode_seq_geom(Lmax, Lmax, window, n_sink, is_full);
+    const SeqGeom longest = decode_seq_geom(Lmax, Lmax, window, n_sink, is_full, paged);
     // upper bound on the tiles of one item: a shorter sequence may have one more (ragged) sink tile
     const long long tiles_ub = (long long)B * Hkv * pl.HG * ((long long)longest.nt + 1);
     long long blocks = (tiles_ub + kDecodeMinTilesPerBlock - 1) / kDecodeMinTilesPerBlock;
@@ -128,13 +128,13 @@ static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, i
     return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
-template <int D, int NH>
+template <int D, int NH, bool kPaged>
 static int launch_decode(const CUtensorMap (&tm)[4], const DecodeParams& p, int blocks, cudaStream_t st) {
     using L = DecodeSmem<D, NH>;
-    if (cudaFuncSetAttribute(decode_kernel<D, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(decode_kernel<D, NH, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             L::kDynamicBytes) != cudaSuccess)
         return SWAA_ERR_CUDA;
-    decode_kernel<D, NH><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tm[0], tm[1], tm[2], tm[3], p);
+    decode_kernel<D, NH, kPaged><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tm[0], tm[1], tm[2], tm[3], p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
@@ -159,29 +159,38 @@ extern "C" int swaa_decode_num_blocks(int B, int Hq, int Hkv, int D, int Lmax, i
     return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count).blocks;
 }
 
-extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
-                           int B, int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
-                           void* workspace, size_t workspace_bytes, void* stream) {
+namespace swaa {
+
+// Shared body of swaa_decode (block_table == nullptr: dense cache [B, Lmax, Hkv, D]) and swaa_decode_paged
+// (cache = pages [num_pages, page_size, Hkv, D]; Lmax = max_blocks * page_size).
+static int decode_impl(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
+                       const int32_t* block_table, int max_blocks, int num_pages, int page_size, int B, int Lmax, int Hq,
+                       int Hkv, int D, int window, int n_sink, int is_full, float scale, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    const bool paged = block_table != nullptr;
     int rc = check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full);
     if (rc != SWAA_OK) return rc;
     if (B == 0) return SWAA_OK;
     if (!q || !kcache || !vcache || !out || !seqlens) return SWAA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(kcache) || !aligned16(vcache) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) != 0) return SWAA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) != 0 || (reinterpret_cast<uintptr_t>(block_table) & 3u) != 0)
+        return SWAA_ERR_INVALID_ARG;
     DeviceInfo info;
     rc = current_device_info(&info);
     if (rc != SWAA_OK) return rc;
     if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
-    const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count);
+    const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count, paged);
     if (pl.too_large) return SWAA_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < pl.bytes)
         return SWAA_ERR_WORKSPACE;
 
-    CUtensorMap tm[4];  // K, V with the full box; K, V with the small box
-    if ((rc = make_cache_map(&tm[0], kcache, B, Lmax, Hkv, D, kDecodeTileKeys)) != SWAA_OK) return rc;
-    if ((rc = make_cache_map(&tm[1], vcache, B, Lmax, Hkv, D, kDecodeTileKeys)) != SWAA_OK) return rc;
-    if ((rc = make_cache_map(&tm[2], kcache, B, Lmax, Hkv, D, kDecodeSmallBoxKeys)) != SWAA_OK) return rc;
-    if ((rc = make_cache_map(&tm[3], vcache, B, Lmax, Hkv, D, kDecodeSmallBoxKeys)) != SWAA_OK) return rc;
+    // K, V with the full box; K, V with the small box.  A paged cache is addressed as (page, row in page).
+    CUtensorMap tm[4];
+    const int outer = paged ? num_pages : B, rows = paged ? page_size : Lmax;
+    if ((rc = make_cache_map(&tm[0], kcache, outer, rows, Hkv, D, kDecodeTileKeys)) != SWAA_OK) return rc;
+    if ((rc = make_cache_map(&tm[1], vcache, outer, rows, Hkv, D, kDecodeTileKeys)) != SWAA_OK) return rc;
+    if ((rc = make_cache_map(&tm[2], kcache, outer, rows, Hkv, D, kDecodeSmallBoxKeys)) != SWAA_OK) return rc;
+    if ((rc = make_cache_map(&tm[3], vcache, outer, rows, Hkv, D, kDecodeSmallBoxKeys)) != SWAA_OK) return rc;
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     DecodeParams p;
@@ -204,9 +213,58 @@ extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache
     p.tickets = reinterpret_cast<unsigned long long*>(ws);
     p.part = reinterpret_cast<float*>(ws + pl.off_part);
     p.stamp = next_call_stamp();
+    p.block_table = block_table;
+    p.max_blocks = max_blocks;
+    p.page_tiles = paged ? page_size / kDecodeTileKeys : 1;
+    p.num_pages = num_pages;
+    if (paged) {
+        if (D == 128)
+            return pl.NH == 1 ? launch_decode<128, 1, true>(tm, p, pl.blocks, st)
+                              : launch_decode<128, 2, true>(tm, p, pl.blocks, st);
+        return pl.NH == 1 ? launch_decode<64, 1, true>(tm, p, pl.blocks, st) : launch_decode<64, 2, true>(tm, p, pl.blocks, st);
+    }
     if (D == 128)
-        return pl.NH == 1 ? launch_decode<128, 1>(tm, p, pl.blocks, st) : launch_decode<128, 2>(tm, p, pl.blocks, st);
-    return pl.NH == 1 ? launch_decode<64, 1>(tm, p, pl.blocks, st) : launch_decode<64, 2>(tm, p, pl.blocks, st);
+        return pl.NH == 1 ? launch_decode<128, 1, false>(tm, p, pl.blocks, st)
+                          : launch_decode<128, 2, false>(tm, p, pl.blocks, st);
+    return pl.NH == 1 ? launch_decode<64, 1, false>(tm, p, pl.blocks, st) : launch_decode<64, 2, false>(tm, p, pl.blocks, st);
+}
+
+static int check_paged_shape(int max_blocks, int num_pages, int page_size) {
+    if (max_blocks < 1 || num_pages < 1 || page_size < 1) return SWAA_ERR_INVALID_ARG;
+    if (page_size % kDecodeTileKeys != 0) return SWAA_ERR_UNSUPPORTED;
+    if ((long long)max_blocks * page_size > 2147483647LL) return SWAA_ERR_UNSUPPORTED;
+    return SWAA_OK;
+}
+
+}  // namespace swaa
+
+extern "C" int swaa_decode(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
+                           int B, int Lmax, int Hq, int Hkv, int D, int window, int n_sink, int is_full, float scale,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_impl(q, kcache, vcache, out, seqlens, nullptr, 0, 0, 0, B, Lmax, Hq, Hkv, D, window, n_sink, is_full,
+                       scale, workspace, workspace_bytes, stream);
+}
+
+extern "C" size_t swaa_decode_paged_workspace_size(int B, int Hq, int Hkv, int D, int max_blocks, int page_size,
+                                                   int window, int n_sink, int is_full) {
+    if (check_paged_shape(max_blocks, 1, page_size) != SWAA_OK) return 256;
+    const int Lmax = max_blocks * page_size;
+    if (check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) != SWAA_OK || B == 0) return 256;
+    DeviceInfo info;
+    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
+    return plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count, true).bytes;
+}
+
+extern "C" int swaa_decode_paged(const void* q, const void* kpages, const void* vpages, void* out,
+                                 const int32_t* block_table, const int32_t* seqlens, int B, int max_blocks,
+                                 int num_pages, int page_size, int Hq, int Hkv, int D, int window, int n_sink,
+                                 int is_full, float scale, void* workspace, size_t workspace_bytes, void* stream) {
+    const int rc = check_paged_shape(max_blocks, num_pages, page_size);
+    if (rc != SWAA_OK) return rc;
+    if (!block_table) return SWAA_ERR_INVALID_ARG;
+    return decode_impl(q, kpages, vpages, out, seqlens, block_table, max_blocks, num_pages, page_size, B,
+                       max_blocks * page_size, Hq, Hkv, D, window, n_sink, is_full, scale, workspace, workspace_bytes,
+                       stream);
 }
 
 // ----------------------------------------------------------------------------------------- prefill

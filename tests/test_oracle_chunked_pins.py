@@ -104,3 +104,30 @@ def test_chunked_rejects_more_queries_than_keys():
     q, k = _bf16_randn((5, 2, 8), 1), _bf16_randn((4, 2, 8), 2)
     with pytest.raises(ValueError):
         oracle.prefill_chunked(q, k, k, [0, 5], [0, 4], 4, 0, False)
+
+
+def test_paged_decode_honours_the_block_table():
+    """A dense cache scattered over pages in random order, unused pages and rows poisoned with NaN."""
+    rng = np.random.default_rng(11)
+    B, Hq, Hkv, D, page = 3, 4, 2, 16, 8
+    sl = [29, 8, 1]
+    max_blocks = 5
+    kc, vc = _bf16_randn((B, max_blocks * page, Hkv, D), 40), _bf16_randn((B, max_blocks * page, Hkv, D), 41)
+    q = _bf16_randn((B, Hq, D), 42)
+    num_pages = 40
+    kp = np.full((num_pages, page, Hkv, D), np.nan, dtype=np.float32)
+    vp = np.full_like(kp, np.nan)
+    perm = rng.permutation(num_pages)
+    bt = np.full((B, max_blocks), -1, dtype=np.int32)
+    nxt = 0
+    for b in range(B):
+        for blk in range((sl[b] + page - 1) // page):
+            pg = perm[nxt]; nxt += 1
+            bt[b, blk] = pg
+            n = min(page, sl[b] - blk * page)
+            kp[pg, :n] = kc[b, blk * page:blk * page + n]
+            vp[pg, :n] = vc[b, blk * page:blk * page + n]
+    for W, S, full in ((6, 2, False), (1, 0, True)):
+        a = oracle.decode_paged(q, kp, vp, bt, sl, W, S, full)
+        d = oracle.decode(q, kc, vc, sl, W, S, full)
+        assert np.array_equal(a["out"], d["out"]) and np.isfinite(a["out"]).all()
