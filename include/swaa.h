@@ -93,6 +93,26 @@ int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out,
                          void* stream);
 
 /*
+ * Lazy ratio of a layer (App. "Results of LightTransfer": layer selection by how much of the attention of the
+ * tokens at the end of a sequence goes to recent tokens rather than to the rest of the context; the paper
+ * uses the last 64 tokens and a recent window of 1024).  For the queries given (the last len_q tokens of each
+ * len_k-token context, packed like swaa_prefill_chunked) and each query head h:
+ *     ratio[h] = mean over the queries of  sum_{j recent or sink} p(i, j),
+ * p = softmax of scale * q.k over ALL keys j <= i (full causal attention), "recent" = the last `recent` keys
+ * ending at the query, "sink" = the first n_sink keys of the sequence.  A value near 1 marks a layer that an SWA
+ * mask would hardly change.  The mass is obtained from two log-sum-exp passes of the prefill kernel (windowed
+ * and full) and a small reduction kernel.
+ *
+ *   ratio        device, float32 [Hq]
+ *   scratch_out  device, bf16 [Tq, Hq, D]; scratch_lse device, float32 [2, Hq, Tq]; both overwritten.
+ * Other arguments, status codes and errors as for swaa_prefill_chunked (recent >= 1, n_sink >= 0).
+ */
+int swaa_lazy_ratio(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_q,
+                    const int32_t* cu_seqlens_k, int B, int Tq, int Tk, int max_seqlen_q, int max_seqlen_k, int Hq,
+                    int Hkv, int D, int recent, int n_sink, float scale, float* ratio, void* scratch_out,
+                    float* scratch_lse, void* stream);
+
+/*
  * Decode: one query token per sequence against a dense KV cache (Sec. 3.1.1 "FA Decode": with is_full
  * the generated token sees the whole context; App. A: the full-context cache is retained).
  *
@@ -206,6 +226,22 @@ int swaa_prefill_block_n(void);
 /* Number of thread blocks swaa_decode cuts the visible cache entries over, for these arguments on the
  * current device (>= 1). */
 int swaa_decode_num_blocks(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full);
+
+/*
+ * Trimmed KV cache of a pure-SWA layer (host only).  App. A: without FA decode an SWA layer never looks
+ * at more than the first n_sink tokens and the last `window` tokens, so its cache can be cut to n_sink + window
+ * entries: the sinks stay in slots 0 .. n_sink-1 and the later tokens go round a ring of `window` slots.
+ *   swaa_trimmed_cache_slot(pos, ...)  slot in which the K/V of the token at position `pos` is stored
+ *   swaa_trimmed_cache_len(len, ...)   occupied slots after `len` tokens = min(len, n_sink + window)
+ * After `len` tokens the occupied slots hold exactly the keys an SWA decode step at that length may see, and
+ * softmax attention does not depend on the order of the keys, so the decode step of such a layer is
+ *   swaa_decode(q, k_trimmed, v_trimmed, out, seqlens = swaa_trimmed_cache_len(len), Lmax = n_sink + window, ...,
+ *               is_full = 1)
+ * and reads the same bytes as swaa_decode with the SWA mask on the untrimmed cache.
+ * Both return -1 on window < 1, n_sink < 0 or a negative position / length.
+ */
+long long swaa_trimmed_cache_slot(long long pos, int window, int n_sink);
+long long swaa_trimmed_cache_len(long long len, int window, int n_sink);
 
 /* Static string for a swaa_status value. */
 const char* swaa_status_str(int status);

@@ -11,6 +11,7 @@ from .swaa_oracle import (  # noqa: F401
     decode,
     decode_paged,
     layer_is_full,
+    lazy_ratio,
     num_threads,
     prefill,
     prefill_chunked,

@@ -198,3 +198,29 @@ def decode_paged(q, kpages, vpages, block_table, seqlens, window: int, n_sink: i
         kd[b, j] = kpages[bt[b, j // page_size], j % page_size]
         vd[b, j] = vpages[bt[b, j // page_size], j % page_size]
     return decode(q, kd, vd, sl, window, n_sink, is_full, scale)
+
+
+def lazy_ratio(q, k, v_unused, cu_seqlens_q, cu_seqlens_k, recent: int, n_sink: int, scale: float | None = None):
+    """Lazy ratio per query head, written out from its definition (App. "Results of LightTransfer"): for every
+    given query (the last len_q tokens of each sequence) the full causal softmax over all keys j <= i, then
+    the share of it that falls on the last `recent` keys ending at the query or on the first n_sink keys;
+    mean over the queries.  Plain float64 numpy loops; v is not needed."""
+    q, k = np.asarray(q, dtype=np.float64), np.asarray(k, dtype=np.float64)
+    Tq, Hq, D = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    cq, ck = np.asarray(cu_seqlens_q, dtype=np.int64), np.asarray(cu_seqlens_k, dtype=np.int64)
+    total = np.zeros(Hq)
+    for b in range(cq.shape[0] - 1):
+        lq, lk = int(cq[b + 1] - cq[b]), int(ck[b + 1] - ck[b])
+        for t in range(lq):
+            i = lk - lq + t
+            keep = np.array([(j > i - recent) or (j < n_sink) for j in range(i + 1)])
+            for h in range(Hq):
+                s = (k[ck[b]:ck[b] + i + 1, h // G] @ q[cq[b] + t, h]) * scale
+                p = np.exp(s - s.max())
+                p /= p.sum()
+                total[h] += p[keep].sum()
+    return total / Tq

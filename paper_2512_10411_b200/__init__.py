@@ -24,7 +24,10 @@ from .binding import (  # noqa: F401
     decode_paged_workspace_size,
     swaa_decode_static,
     DECODE_STATIC_SCRATCH_BYTES,
+    swaa_lazy_ratio,
     swaa_prefill,
     swaa_prefill_chunked,
     last_device_status,
+    trimmed_cache_len,
+    trimmed_cache_slot,
 )

@@ -64,6 +64,8 @@ def load_library():
     lib.swaa_prefill.restype = ci
     lib.swaa_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     lib.swaa_prefill_chunked.restype = ci
+    lib.swaa_lazy_ratio.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
+    lib.swaa_lazy_ratio.restype = ci
     lib.swaa_decode_workspace_size.argtypes = [ci] * 8
     lib.swaa_decode_workspace_size.restype = ctypes.c_size_t
     lib.swaa_decode_num_blocks.argtypes = [ci] * 8
@@ -86,6 +88,10 @@ def load_library():
     lib.swaa_prefill_tile_needs_mask.restype = ci
     lib.swaa_prefill_block_m.restype = ci
     lib.swaa_prefill_block_n.restype = ci
+    lib.swaa_trimmed_cache_slot.argtypes = [ctypes.c_longlong, ci, ci]
+    lib.swaa_trimmed_cache_slot.restype = ctypes.c_longlong
+    lib.swaa_trimmed_cache_len.argtypes = [ctypes.c_longlong, ci, ci]
+    lib.swaa_trimmed_cache_len.restype = ctypes.c_longlong
     lib.swaa_status_str.argtypes = [ci]
     lib.swaa_status_str.restype = ctypes.c_char_p
     lib.swaa_last_device_status.argtypes = [vp]
@@ -161,6 +167,27 @@ def swaa_prefill_chunked(q, k, v, out, cu_seqlens_q, cu_seqlens_k, max_seqlen_q:
         raise SwaaError(rc, "swaa_prefill_chunked")
 
 
+def swaa_lazy_ratio(q, k, v, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, recent: int, n_sink: int,
+                    ratio, scratch_out, scratch_lse, scale: float = 0.0, stream=None) -> None:
+    """Forwards to C swaa_lazy_ratio.  q [Tq,Hq,D]; k, v [Tk,Hkv,D] bf16; ratio f32 [Hq]; scratch_out bf16 [Tq,Hq,D];
+    scratch_lse f32 [2,Hq,Tq]."""
+    lib = load_library()
+    Tq, Hq, D = q.shape
+    Tk, Hkv = k.shape[0], k.shape[1]
+    if tuple(scratch_out.shape) != (Tq, Hq, D) or tuple(scratch_lse.shape) != (2, Hq, Tq) or tuple(ratio.shape) != (Hq,):
+        raise ValueError("swaa_lazy_ratio: inconsistent output / scratch shapes")
+    B = cu_seqlens_q.numel() - 1
+    bf = torch.bfloat16
+    rc = lib.swaa_lazy_ratio(_dev_ptr(q, bf, "q"), _dev_ptr(k, bf, "k"), _dev_ptr(v, bf, "v"),
+                             _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
+                             _dev_ptr(cu_seqlens_k, torch.int32, "cu_seqlens_k"), B, Tq, Tk, int(max_seqlen_q),
+                             int(max_seqlen_k), Hq, Hkv, D, int(recent), int(n_sink), float(scale),
+                             _dev_ptr(ratio, torch.float32, "ratio"), _dev_ptr(scratch_out, bf, "scratch_out"),
+                             _dev_ptr(scratch_lse, torch.float32, "scratch_lse"), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_lazy_ratio")
+
+
 def decode_workspace_size(B, Hq, Hkv, D, Lmax, window, n_sink, is_full) -> int:
     """Forwards to C swaa_decode_workspace_size (bytes)."""
     return int(load_library().swaa_decode_workspace_size(B, Hq, Hkv, D, Lmax, int(window), int(n_sink),
@@ -216,6 +243,16 @@ def swaa_decode_paged(q, kpages, vpages, out, block_table, seqlens, window: int,
                                _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_decode_paged")
+
+
+def trimmed_cache_slot(pos: int, window: int, n_sink: int) -> int:
+    """Forwards to C swaa_trimmed_cache_slot."""
+    return int(load_library().swaa_trimmed_cache_slot(int(pos), int(window), int(n_sink)))
+
+
+def trimmed_cache_len(length: int, window: int, n_sink: int) -> int:
+    """Forwards to C swaa_trimmed_cache_len."""
+    return int(load_library().swaa_trimmed_cache_len(int(length), int(window), int(n_sink)))
 
 
 DECODE_STATIC_SCRATCH_BYTES = 2 << 20

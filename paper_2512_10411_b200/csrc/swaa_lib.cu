@@ -383,6 +383,49 @@ extern "C" int swaa_prefill_chunked(const void* q, const void* k, const void* v,
                         window, n_sink, is_full, scale, lse, stream);
 }
 
+// ------------------------------------------------------------------------------------ lazy ratio
+namespace swaa {
+
+// ratio[h] = mean over t of exp(lse_recent[h, t] - lse_full[h, t]); one block per head.
+__global__ void lazy_ratio_reduce_kernel(const float* __restrict__ lse_recent, const float* __restrict__ lse_full,
+                                         int Tq, float* __restrict__ ratio) {
+    __shared__ float warp_sums[8];
+    const int h = blockIdx.x;
+    float acc = 0.f;
+    for (int t = threadIdx.x; t < Tq; t += blockDim.x)
+        acc += __expf(lse_recent[(size_t)h * Tq + t] - lse_full[(size_t)h * Tq + t]);
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float total = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) total += warp_sums[w];
+        ratio[h] = total / (float)Tq;
+    }
+}
+
+}  // namespace swaa
+
+extern "C" int swaa_lazy_ratio(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_q,
+                               const int32_t* cu_seqlens_k, int B, int Tq, int Tk, int max_seqlen_q, int max_seqlen_k,
+                               int Hq, int Hkv, int D, int recent, int n_sink, float scale, float* ratio,
+                               void* scratch_out, float* scratch_lse, void* stream) {
+    if (!ratio || !scratch_out || !scratch_lse || !cu_seqlens_k) return SWAA_ERR_INVALID_ARG;
+    if (recent < 1 || B < 1 || Tq < 1) return SWAA_ERR_INVALID_ARG;
+    float* lse_recent = scratch_lse;
+    float* lse_full = scratch_lse + (size_t)Hq * Tq;
+    int rc = prefill_impl(q, k, v, scratch_out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq,
+                          Hkv, D, recent, n_sink, 0, scale, lse_recent, stream);
+    if (rc != SWAA_OK) return rc;
+    rc = prefill_impl(q, k, v, scratch_out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq, Hkv, D,
+                      1, 0, 1, scale, lse_full, stream);
+    if (rc != SWAA_OK) return rc;
+    lazy_ratio_reduce_kernel<<<(unsigned)Hq, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(lse_recent, lse_full, Tq,
+                                                                                                ratio);
+    launch_counter().fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------- decode without allocation
 namespace swaa {
 
@@ -448,6 +491,18 @@ extern "C" int swaa_schedule_fill(const swaa_policy* policy, int phase, uint8_t*
         is_full_out[l] = (uint8_t)r;
     }
     return SWAA_OK;
+}
+
+// -------------------------------------------------------------------------------- trimmed cache
+extern "C" long long swaa_trimmed_cache_slot(long long pos, int window, int n_sink) {
+    if (window < 1 || n_sink < 0 || pos < 0) return -1;
+    return pos < n_sink ? pos : (long long)n_sink + (pos - n_sink) % window;
+}
+
+extern "C" long long swaa_trimmed_cache_len(long long len, int window, int n_sink) {
+    if (window < 1 || n_sink < 0 || len < 0) return -1;
+    const long long cap = (long long)n_sink + window;
+    return len < cap ? len : cap;
 }
 
 // ------------------------------------------------------------------------------- tile enumeration

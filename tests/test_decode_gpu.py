@@ -167,3 +167,24 @@ def test_decode_full_size_workload(full):
         r = check_against_oracle(out[b:b + 4], ref["out"], f"cfg4 full={full} b={b}")
         worst = max(worst, r)
     print(f"cfg4 decode full={full}: max abs err {worst[0]:.3e}, max rel err {worst[1]:.3e}")
+
+
+def test_decode_on_a_trimmed_ring_cache_equals_swa_decode():
+    """A pure-SWA layer keeps n_sink + window cache entries (ring); full attention over them is the SWA decode."""
+    B, Hq, Hkv, D, W, S = 3, 8, 2, 128, 200, 5
+    sl = (1000, 150, 206)
+    cfg = inputs.DecodeConfig("t", B, 1000, Hq, Hkv, D, W, S, seed=55, seqlens=sl)
+    q, kc, vc, seqlens = inputs.make_decode_inputs(cfg, "cuda")
+    cap = S + W
+    kt = torch.full((B, cap, Hkv, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vt = torch.full_like(kt, float("nan"))
+    for b, n in enumerate(sl):
+        for pos in range(n):  # the order in which a serving loop would append
+            slot = swaa.trimmed_cache_slot(pos, W, S)
+            kt[b, slot] = kc[b, pos]
+            vt[b, slot] = vc[b, pos]
+    tl = torch.tensor([swaa.trimmed_cache_len(n, W, S) for n in sl], dtype=torch.int32, device="cuda")
+    out, status = _run_decode(q, kt, vt, tl, 1, 0, True)
+    assert status == 0
+    ref = oracle.decode(inputs.to_f32_numpy(q), inputs.to_f32_numpy(kc), inputs.to_f32_numpy(vc), sl, W, S, False)
+    check_against_oracle(out, ref["out"], "trimmed ring cache")

@@ -125,3 +125,22 @@ def test_decode_split_plan_is_consistent():
         assert swaa.decode_workspace_size(*args) >= 8 * nb + 2 * nb * heads * (D + 2) * 4
     # a problem of a single tile needs a single block
     assert swaa.decode_num_blocks(1, 4, 2, 64, 100, 8, 0, 0) == 1
+
+
+def test_trimmed_cache_holds_exactly_the_visible_keys():
+    """Appending tokens 0 .. len-1 into the trimmed cache leaves, in its occupied slots, exactly the positions
+    the oracle's SWA predicate shows to the decode query at position len-1 (App. A)."""
+    for W, S in ((1, 0), (4, 0), (4, 3), (5, 9), (16, 2), (3, 1)):
+        cap = S + W
+        slots = {}
+        for n in range(1, 60):
+            pos = n - 1
+            slot = swaa.trimmed_cache_slot(pos, W, S)
+            assert 0 <= slot < cap
+            slots[slot] = pos
+            used = swaa.trimmed_cache_len(n, W, S)
+            assert used == min(n, cap) == len(slots)
+            assert sorted(slots) == list(range(used))  # occupied slots are a prefix: seqlens = used addresses them
+            want = {j for j in range(n) if oracle.visible(n - 1, j, W, S, False)}
+            assert set(slots.values()) == want, (W, S, n)
+    assert swaa.trimmed_cache_slot(-1, 4, 0) == -1 and swaa.trimmed_cache_len(5, 0, 0) == -1

@@ -131,3 +131,33 @@ def test_paged_decode_honours_the_block_table():
         a = oracle.decode_paged(q, kp, vp, bt, sl, W, S, full)
         d = oracle.decode(q, kc, vc, sl, W, S, full)
         assert np.array_equal(a["out"], d["out"]) and np.isfinite(a["out"]).all()
+
+
+def test_lazy_ratio_closed_forms():
+    """Q = 0 makes the softmax uniform: the share of the recent and sink keys is a count ratio.  A recent window
+    that covers the whole context gives 1.  Scores that single out one old key give (almost) 0."""
+    Hq, Hkv, D, lq, lk, recent, S = 4, 2, 16, 5, 40, 8, 3
+    k = _bf16_randn((lk, Hkv, D), 50)
+    q0 = np.zeros((lq, Hq, D), dtype=np.float32)
+    r = oracle.lazy_ratio(q0, k, None, [0, lq], [0, lk], recent, S)
+    want = np.mean([(recent + S) / (lk - lq + t + 1) for t in range(lq)])
+    assert np.allclose(r, want, atol=1e-12)
+    q = _bf16_randn((lq, Hq, D), 51)
+    assert np.allclose(oracle.lazy_ratio(q, k, None, [0, lq], [0, lk], 1000, 0), 1.0, atol=1e-12)
+    kk = np.zeros((lk, Hkv, D), dtype=np.float32)
+    kk[10, :, 0] = 100.0  # key 10 is far outside the recent window of the last queries and not a sink
+    qq = np.zeros((lq, Hq, D), dtype=np.float32)
+    qq[:, :, 0] = 10.0
+    assert (oracle.lazy_ratio(qq, kk, None, [0, lq], [0, lk], recent, S, scale=1.0) < 1e-300).all()
+
+
+def test_lazy_ratio_equals_mass_from_two_log_sum_exps():
+    """Independent route: exp(lse over recent+sink keys - lse over all keys) from the attention oracle."""
+    Hq, Hkv, D, recent, S = 4, 2, 16, 6, 2
+    lq, lk = [3, 4], [30, 9]
+    cq, ck = np.concatenate([[0], np.cumsum(lq)]), np.concatenate([[0], np.cumsum(lk)])
+    q, k = _bf16_randn((sum(lq), Hq, D), 60), _bf16_randn((sum(lk), Hkv, D), 61)
+    v = _bf16_randn((sum(lk), Hkv, D), 62)
+    a = oracle.prefill_chunked(q, k, v, cq, ck, recent, S, False)["lse"]
+    b = oracle.prefill_chunked(q, k, v, cq, ck, 1, 0, True)["lse"]
+    assert np.allclose(oracle.lazy_ratio(q, k, v, cq, ck, recent, S), np.exp(a - b).mean(axis=0), atol=1e-12)

@@ -123,3 +123,20 @@ def test_chunked_prefill_reports_more_queries_than_keys():
                                  [0, 64], [0, 80], 16, 0, False)
     check_against_oracle(out[:64], ref["out"], "valid sequence next to a bad one")
     assert torch.isnan(out[64:].float()).all()  # rows of the bad sequence are not written
+
+
+def test_lazy_ratio_matches_oracle():
+    """Last 64 tokens of two contexts, recent window 1024 (the paper's probe), plus a small ragged case."""
+    for lq, lk, Hq, Hkv, D, recent, S in (((64, 64), (3000, 1500), 8, 2, 128, 1024, 0), ((5, 64), (70, 900), 4, 2, 64, 100, 4)):
+        q, k, v = make(lq, lk, Hq, Hkv, D, seed=123)
+        q = (q.float() * 2.0).to(torch.bfloat16)  # sharper softmax: the ratio is not just a key count
+        ratio = torch.full((Hq,), float("nan"), device="cuda")
+        so = torch.empty_like(q)
+        sl = torch.empty((2, Hq, sum(lq)), dtype=torch.float32, device="cuda")
+        swaa.swaa_lazy_ratio(q, k, v, _cu(lq), _cu(lk), max(lq), max(lk), recent, S, ratio, so, sl)
+        assert swaa.last_device_status() == 0
+        ref = oracle.lazy_ratio(inputs.to_f32_numpy(q), inputs.to_f32_numpy(k), None, _cu(lq).cpu().numpy(),
+                                _cu(lk).cpu().numpy(), recent, S)
+        got = ratio.cpu().numpy()
+        assert np.abs(got - ref).max() <= 5e-3, (got, ref)
+        assert ((ref > 0.05) & (ref < 0.999)).any()
