@@ -165,6 +165,24 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, world, device=None):
+    """Every rank runs the same independent problem (replicas, no collective on the data path); a timing of
+    the job is the slowest rank's.  Returns the element-wise maximum over ranks of `values` on every rank."""
+    import torch
+
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(units_per_rank, n_ranks, seconds):
+    """Throughput of the whole job: the units all ranks processed over the slowest rank's time."""
+    return n_ranks * units_per_rank / seconds
+
+
 def run_ours(args, rank, local_rank, world):
     import numpy as np
     import torch
@@ -299,10 +317,8 @@ def run_ours(args, rank, local_rank, world):
     e2e_swa_ms = time_loop(lambda: e2e_decode_step(False, ws_swa), e2e_steps)
 
     # ---------------------------------------------------------------- max over ranks
-    times = torch.tensor([total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms = times.tolist()
+    total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms = max_over_ranks(
+        [total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms], world, dev)
     K, N = args.steps, world
 
     cpu_baseline = None
@@ -330,7 +346,7 @@ def run_ours(args, rank, local_rank, world):
             dist.destroy_process_group()
         return
     avg_pre_ms = t_pre / K
-    achieved = prefill_flops / (avg_pre_ms * 1e-3) / 1e12
+    achieved = whole_job_value(prefill_flops, 1, avg_pre_ms * 1e-3) / 1e12  # per GPU; the line reports N x this
     fa_gbs = fa_bytes / (t_fa / K * 1e-3) / 1e9
     swa_gbs = swa_bytes / (t_swa / K * 1e-3) / 1e9
     line = {

@@ -1,0 +1,55 @@
+"""The N > 1 path of bench.py on CPU: two gloo ranks on 127.0.0.1.  The path shards without any exchange
+(every rank runs an independent replica), so all there is to test is the timing reduction (max over ranks),
+the whole-job throughput, and that the reference arm prints from rank 0 only."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = r"""
+import os, sys, json
+sys.path.insert(0, os.environ["SWAA_ROOT"])
+import torch.distributed as dist
+import bench
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+mine = [10.0 + rank, 5.0 - rank, 1.0]            # per-rank timings: rank 1 is slower on the first, faster on the second
+red = bench.max_over_ranks(mine, world)
+value = bench.whole_job_value(100.0, world, red[0])
+print(json.dumps({"rank": rank, "red": red, "value": value}), flush=True)
+dist.destroy_process_group()
+"""
+
+
+def _launch(args, env_extra=None, timeout=300):
+    env = dict(os.environ, SWAA_ROOT=ROOT, MASTER_ADDR="127.0.0.1", **(env_extra or {}))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
+           "127.0.0.1", "--master-port", "29531"] + args
+    return subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=timeout, cwd=ROOT)
+
+
+def test_two_rank_timing_reduction(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER)
+    r = _launch([str(script)])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert sorted(d["rank"] for d in lines) == [0, 1]
+    for d in lines:
+        assert d["red"] == [11.0, 5.0, 1.0]                # element-wise max over the two ranks, on every rank
+        assert d["value"] == pytest.approx(2 * 100.0 / 11.0)  # units of all ranks over the slowest rank's time
+
+
+def test_reference_arm_prints_from_rank_zero_only():
+    r = _launch(["bench.py", "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0"],
+                env_extra={"OMP_NUM_THREADS": "2"}, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = lines[0]
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["value"] > 0
