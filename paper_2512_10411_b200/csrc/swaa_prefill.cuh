@@ -150,7 +150,7 @@ __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, floa
 
 // Bit c (0..15) set: column pair c of every 32-column chunk of a score tile takes the polynomial path.
 #ifndef SWAA_POLY_PAIR_MASK
-#define SWAA_POLY_PAIR_MASK 0x8888u
+#define SWAA_POLY_PAIR_MASK 0x8080u
 #endif
 constexpr uint32_t kPolyPairMask = SWAA_POLY_PAIR_MASK;
 
