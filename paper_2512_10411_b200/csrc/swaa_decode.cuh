@@ -558,40 +558,67 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             // ---- the last block of this item to arrive merges the item's partials
             const long long T0 = seg_t0 - ti_begin, T1 = T0 + nt;
             const int c_first = (int)(T0 / tpc), c_last = (int)((T1 - 1) / tpc);
-            __threadfence();
+            const int n_parts = c_last - c_first + 1;
+            __threadfence();  // this block's partial is visible before its ticket
             consumer_sync();
             if (tid == 0) {
                 // A ticket whose stamp is not this call's is left over from an earlier call (or was never
                 // written): the first block to arrive restarts it, so the workspace needs no clearing.
                 unsigned long long* t = p.tickets + c_first;
-                unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(t), want;
-                for (;;) {
-                    want = (seen >> 16) == p.stamp ? seen + 1ull : ((p.stamp << 16) | 1ull);
-                    const unsigned long long prev = atomicCAS(t, seen, want);
-                    if (prev == seen) break;
-                    seen = prev;
+                if (n_parts == 2) {
+                    // two blocks share the item (the common case): one exchange tells who came second
+                    const unsigned long long mine = (p.stamp << 16) | 1ull;
+                    *sm_last = atomicExch(t, mine) == mine ? 1 : 0;
+                } else {
+                    unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(t), want;
+                    for (;;) {
+                        want = (seen >> 16) == p.stamp ? seen + 1ull : ((p.stamp << 16) | 1ull);
+                        const unsigned long long prev = atomicCAS(t, seen, want);
+                        if (prev == seen) break;
+                        seen = prev;
+                    }
+                    *sm_last = ((int)(want & 0xffffull) == n_parts) ? 1 : 0;
                 }
-                *sm_last = ((int)(want & 0xffffull) == c_last - c_first + 1) ? 1 : 0;
             }
             consumer_sync();
             if (*sm_last && ok) {
                 __threadfence();
                 const bool first_is_slot1 = (long long)c_first * tpc != T0;
+                auto slot_of = [&](int cc) { return 2 * cc + ((cc == c_first && first_is_slot1) ? 1 : 0); };
                 for (int idx = tid; idx < gc * D; idx += kDecodeConsumerThreads) {
                     const int hh = idx / D, d = idx - hh * D;
-                    float M = -INFINITY;
-                    for (int cc = c_first; cc <= c_last; ++cc) {
-                        const int sl = 2 * cc + ((cc == c_first && first_is_slot1) ? 1 : 0);
-                        M = fmaxf(M, __ldcg(p.part + ((size_t)sl * HC + hh) * (D + 2)));
-                    }
-                    float den = 0.f, num = 0.f;
-                    for (int cc = c_first; cc <= c_last; ++cc) {
-                        const int sl = 2 * cc + ((cc == c_first && first_is_slot1) ? 1 : 0);
-                        const float* pp = p.part + ((size_t)sl * HC + hh) * (D + 2);
-                        const float ms = __ldcg(pp);
-                        const float wgt = ms == -INFINITY ? 0.f : ex2f((ms - M) * p.sl2);
-                        den += wgt * __ldcg(pp + 1);
-                        num += wgt * __ldcg(pp + 2 + d);
+                    float M = -INFINITY, den = 0.f, num = 0.f;
+                    if (n_parts <= 4) {
+                        // few parts: every load is issued before the first is needed (one round trip to L2)
+                        float ms[4], ls[4], os[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            ms[i] = -INFINITY;
+                            ls[i] = os[i] = 0.f;
+                            if (i < n_parts) {
+                                const float* pp = p.part + ((size_t)slot_of(c_first + i) * HC + hh) * (D + 2);
+                                ms[i] = __ldcg(pp);
+                                ls[i] = __ldcg(pp + 1);
+                                os[i] = __ldcg(pp + 2 + d);
+                            }
+                        }
+                        M = fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3]));
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float wgt = ms[i] == -INFINITY ? 0.f : ex2f((ms[i] - M) * p.sl2);
+                            den += wgt * ls[i];
+                            num += wgt * os[i];
+                        }
+                    } else {
+                        for (int cc = c_first; cc <= c_last; ++cc)
+                            M = fmaxf(M, __ldcg(p.part + ((size_t)slot_of(cc) * HC + hh) * (D + 2)));
+                        for (int cc = c_first; cc <= c_last; ++cc) {
+                            const float* pp = p.part + ((size_t)slot_of(cc) * HC + hh) * (D + 2);
+                            const float ms = __ldcg(pp);
+                            const float wgt = ms == -INFINITY ? 0.f : ex2f((ms - M) * p.sl2);
+                            den += wgt * __ldcg(pp + 1);
+                            num += wgt * __ldcg(pp + 2 + d);
+                        }
                     }
                     p.out[((size_t)b * p.Hq + h0 + hh) * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
                 }
