@@ -496,7 +496,34 @@ def run_sweep():
         print(json.dumps({"case": "chunked_prefill", "len_q": lq, "len_k": lk, "Hq": Hq, "Hkv": Hkv, "D": D, "window": W,
                           "n_sink": S, "is_full": full, "ms": ms[len(ms) // 2], "effective_tflops": tf,
                           "frac_of_measured_peak": tf / peaks["bf16_tflops"]}), flush=True)
-    del cq, ck, cv, cout
+    # the same chunk against a paged pool (256-entry pages in random order)
+    pg = 256
+    nb = lk // pg
+    perm = torch.randperm(nb, generator=g, device="cuda")
+    pkp = torch.empty((nb, pg, Hkv, D), dtype=torch.bfloat16, device="cuda")
+    pvp = torch.empty_like(pkp)
+    pkp[perm] = ck.view(nb, pg, Hkv, D)
+    pvp[perm] = cv.view(nb, pg, Hkv, D)
+    pbt = perm.view(1, nb).to(torch.int32).contiguous()
+    psk = torch.tensor([lk], dtype=torch.int32, device="cuda")
+    ms = []
+    for r in range(6):
+        flush.zero_()
+        flush_rd.sum()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        swaa.swaa_prefill_paged(cq, pkp, pvp, cout, cuq, psk, pbt, lq, W, S, False)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if r > 0:
+            ms.append(a.elapsed_time(b))
+    assert swaa.last_device_status() == 0
+    ms.sort()
+    tf = 4.0 * D * Hq * lq * (W + S) / (ms[len(ms) // 2] * 1e-3) / 1e12
+    print(json.dumps({"case": "paged_chunked_prefill", "len_q": lq, "len_k": lk, "page_size": pg, "window": W, "n_sink": S,
+                      "is_full": False, "ms": ms[len(ms) // 2], "effective_tflops": tf,
+                      "frac_of_measured_peak": tf / peaks["bf16_tflops"]}), flush=True)
+    del cq, ck, cv, cout, pkp, pvp
     # paged decode: workload 4 with 256-entry pages handed out in random order, against the dense layout
     dcfg = inputs.cfg_decode()
     dq, kc, vc, sl = inputs.make_decode_inputs(dcfg, "cuda")

@@ -93,6 +93,24 @@ int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out,
                          void* stream);
 
 /*
+ * Chunked prefill against a paged KV cache (the two needs of a serving engine that mixes prefill chunks and
+ * decode steps, Sec. 4.1.1): queries as in swaa_prefill_chunked, keys and values as in swaa_decode_paged.
+ *
+ *   q, out          device, [Tq, Hq, D] bf16, packed by cu_seqlens_q (int32 [B+1])
+ *   kpages, vpages  device, [num_pages, page_size, Hkv, D] bf16; page_size is a multiple of 128.
+ *   seqlens_k       device, int32 [B]; keys of sequence b INCLUDING the chunk's own tokens, len_q <= len_k <=
+ *                   max_blocks * page_size.
+ *   block_table     device, int32 [B, max_blocks]; entry j of sequence b lives in page
+ *                   block_table[b][j / page_size] at row j % page_size.
+ * The rows of a page past a sequence's last key are never used, whatever they hold.  A page index outside
+ * [0, num_pages) or len_q > len_k is reported as SWAA_ERR_BAD_SEQLENS through the status word.
+ */
+int swaa_prefill_paged(const void* q, const void* kpages, const void* vpages, void* out, const int32_t* cu_seqlens_q,
+                       const int32_t* seqlens_k, const int32_t* block_table, int B, int Tq, int max_seqlen_q,
+                       int max_blocks, int num_pages, int page_size, int Hq, int Hkv, int D, int window, int n_sink,
+                       int is_full, float scale, float* lse, void* stream);
+
+/*
  * Lazy ratio of a layer (App. "Results of LightTransfer": layer selection by how much of the attention of the
  * tokens at the end of a sequence goes to recent tokens rather than to the rest of the context; the paper
  * uses the last 64 tokens and a recent window of 1024).  For the queries given (the last len_q tokens of each

@@ -15,5 +15,6 @@ from .swaa_oracle import (  # noqa: F401
     num_threads,
     prefill,
     prefill_chunked,
+    prefill_paged,
     visible,
 )

@@ -224,3 +224,21 @@ def lazy_ratio(q, k, v_unused, cu_seqlens_q, cu_seqlens_k, recent: int, n_sink: 
                 p /= p.sum()
                 total[h] += p[keep].sum()
     return total / Tq
+
+
+def prefill_paged(q, kpages, vpages, cu_seqlens_q, seqlens_k, block_table, window: int, n_sink: int, is_full: bool,
+                  scale: float | None = None, rows=None):
+    """Chunked prefill against a paged cache, by definition: the keys and values of each sequence are gathered
+    from their pages (pure indexing) into the packed layout and handed to prefill_chunked."""
+    kpages, vpages = _f32(kpages), _f32(vpages)
+    bt = np.asarray(block_table, dtype=np.int64)
+    lk = np.asarray(seqlens_k, dtype=np.int64)
+    page_size = kpages.shape[1]
+    ks, vs = [], []
+    for b in range(bt.shape[0]):
+        j = np.arange(int(lk[b]))
+        ks.append(kpages[bt[b, j // page_size], j % page_size])
+        vs.append(vpages[bt[b, j // page_size], j % page_size])
+    cu_k = np.concatenate([[0], np.cumsum(lk)])
+    return prefill_chunked(q, np.concatenate(ks), np.concatenate(vs), cu_seqlens_q, cu_k, window, n_sink, is_full, scale,
+                           rows)

@@ -27,6 +27,7 @@ from .binding import (  # noqa: F401
     swaa_lazy_ratio,
     swaa_prefill,
     swaa_prefill_chunked,
+    swaa_prefill_paged,
     last_device_status,
     trimmed_cache_len,
     trimmed_cache_slot,

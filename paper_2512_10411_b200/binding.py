@@ -64,6 +64,8 @@ def load_library():
     lib.swaa_prefill.restype = ci
     lib.swaa_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     lib.swaa_prefill_chunked.restype = ci
+    lib.swaa_prefill_paged.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
+    lib.swaa_prefill_paged.restype = ci
     lib.swaa_lazy_ratio.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
     lib.swaa_lazy_ratio.restype = ci
     lib.swaa_decode_workspace_size.argtypes = [ci] * 8
@@ -165,6 +167,32 @@ def swaa_prefill_chunked(q, k, v, out, cu_seqlens_q, cu_seqlens_k, max_seqlen_q:
                                   float(scale), _dev_ptr(lse, torch.float32, "lse"), _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_prefill_chunked")
+
+
+def swaa_prefill_paged(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, block_table, max_seqlen_q: int, window: int,
+                       n_sink: int, is_full: bool, scale: float = 0.0, lse=None, stream=None) -> None:
+    """Forwards to C swaa_prefill_paged.  q, out [Tq,Hq,D]; kpages, vpages [num_pages,page_size,Hkv,D] bf16;
+    cu_seqlens_q int32 [B+1]; seqlens_k int32 [B]; block_table int32 [B,max_blocks]; lse f32 [Hq,Tq]."""
+    lib = load_library()
+    Tq, Hq, D = q.shape
+    num_pages, page_size, Hkv, _ = kpages.shape
+    if tuple(vpages.shape) != tuple(kpages.shape) or kpages.shape[3] != D or tuple(out.shape) != (Tq, Hq, D):
+        raise ValueError("swaa_prefill_paged: inconsistent tensor shapes")
+    B = cu_seqlens_q.numel() - 1
+    if block_table.dim() != 2 or block_table.shape[0] != B or seqlens_k.numel() != B:
+        raise ValueError("swaa_prefill_paged: block_table must be [B, max_blocks] and seqlens_k [B]")
+    if lse is not None and tuple(lse.shape) != (Hq, Tq):
+        raise ValueError("swaa_prefill_paged: lse must be [Hq, Tq]")
+    bf = torch.bfloat16
+    rc = lib.swaa_prefill_paged(_dev_ptr(q, bf, "q"), _dev_ptr(kpages, bf, "kpages"), _dev_ptr(vpages, bf, "vpages"),
+                                _dev_ptr(out, bf, "out"), _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
+                                _dev_ptr(seqlens_k, torch.int32, "seqlens_k"),
+                                _dev_ptr(block_table, torch.int32, "block_table"), B, Tq, int(max_seqlen_q),
+                                block_table.shape[1], num_pages, page_size, Hq, Hkv, D, int(window), int(n_sink),
+                                int(bool(is_full)), float(scale), _dev_ptr(lse, torch.float32, "lse"),
+                                _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_prefill_paged")
 
 
 def swaa_lazy_ratio(q, k, v, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, recent: int, n_sink: int,

@@ -188,7 +188,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     __shared__ int sc_b0;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef SWAA_DECODE_REVERSE_BLOCKS  // development aid: hand the runs of the tile list out in reverse block order
+    const int ncta = (int)gridDim.x, cta = (int)(gridDim.x - 1 - blockIdx.x);
+#else
     const int ncta = (int)gridDim.x, cta = (int)blockIdx.x;
+#endif
     if (warp == 0) SWAA_DSTAMP(0);  // block entered
 
     if (tid == 0) {

@@ -285,17 +285,17 @@ static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H
     return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
-template <int D, bool kChunked>
+template <int D, int kMode>
 static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                           const PrefillParams& p, int sm_count, cudaStream_t st) {
     using L = PrefillSmem<D>;
-    if (cudaFuncSetAttribute(prefill_kernel<D, kChunked>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(prefill_kernel<D, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              L::kDynamicBytes) != cudaSuccess)
         return SWAA_ERR_CUDA;
     // persistent blocks: one per SM (or fewer when there is less work), each walks its share of the items
     long long blocks = (long long)p.n_pairs * p.tiles_ub;
     if (blocks > sm_count) blocks = sm_count;
-    prefill_kernel<D, kChunked><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, p);
+    prefill_kernel<D, kMode><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
@@ -306,9 +306,15 @@ namespace swaa {
 
 // Shared body of swaa_prefill (cu_seqlens_k == nullptr: keys are packed like the queries) and
 // swaa_prefill_chunked.
+struct PagedKV {  // keys and values in pages (null block_table: packed layout)
+    const int32_t* block_table = nullptr;
+    int max_blocks = 0, num_pages = 0, page_size = 0;
+};
+
 static int prefill_impl(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens_q,
                         const int32_t* cu_seqlens_k, int B, int Tq, int Tk, int max_seqlen_q, int max_seqlen_k, int Hq,
-                        int Hkv, int D, int window, int n_sink, int is_full, float scale, float* lse, void* stream) {
+                        int Hkv, int D, int window, int n_sink, int is_full, float scale, float* lse, void* stream,
+                        const PagedKV& paged = PagedKV()) {
     if (B < 0 || Tq < 0 || Tk < 0 || max_seqlen_q < 0 || max_seqlen_k < 0 || Hq < 1 || Hkv < 1 || n_sink < 0)
         return SWAA_ERR_INVALID_ARG;
     if (!is_full && window < 1) return SWAA_ERR_INVALID_ARG;
@@ -319,7 +325,8 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
     if ((reinterpret_cast<uintptr_t>(cu_seqlens_q) & 3u) != 0 || (reinterpret_cast<uintptr_t>(cu_seqlens_k) & 3u) != 0 ||
         (reinterpret_cast<uintptr_t>(lse) & 3u) != 0)
         return SWAA_ERR_INVALID_ARG;
-    if (Tk < Tq) return SWAA_ERR_INVALID_ARG;
+    const bool is_paged = paged.block_table != nullptr;
+    if (!is_paged && Tk < Tq) return SWAA_ERR_INVALID_ARG;
     DeviceInfo info;
     int rc = current_device_info(&info);
     if (rc != SWAA_OK) return rc;
@@ -327,8 +334,13 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
 
     CUtensorMap tq, tk, tv, to;
     if ((rc = make_token_major_map(&tq, q, Tq, Hq, D)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&tk, k, Tk, Hkv, D)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&tv, v, Tk, Hkv, D)) != SWAA_OK) return rc;
+    if (is_paged) {  // (D, Hkv, page_size, num_pages), boxes of 128 rows of one page
+        if ((rc = make_cache_map(&tk, k, paged.num_pages, paged.page_size, Hkv, D, kPrefillBN)) != SWAA_OK) return rc;
+        if ((rc = make_cache_map(&tv, v, paged.num_pages, paged.page_size, Hkv, D, kPrefillBN)) != SWAA_OK) return rc;
+    } else {
+        if ((rc = make_token_major_map(&tk, k, Tk, Hkv, D)) != SWAA_OK) return rc;
+        if ((rc = make_token_major_map(&tv, v, Tk, Hkv, D)) != SWAA_OK) return rc;
+    }
     if ((rc = make_token_major_map(&to, out, Tq, Hq, D, 32)) != SWAA_OK) return rc;  // output rows, 32 at a time
 
     PrefillParams p;
@@ -341,6 +353,10 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
     p.Tk = Tk;
     p.max_seqlen = max_seqlen_q;
     p.max_seqlen_k = max_seqlen_k;
+    p.block_table = paged.block_table;
+    p.max_blocks = paged.max_blocks;
+    p.page_size = paged.page_size;
+    p.num_pages = paged.num_pages;
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.G = Hq / Hkv;
@@ -358,11 +374,14 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
     p.sl2 = p.scale * 1.4426950408889634f;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (is_paged)
+        return D == 128 ? launch_prefill<128, 2>(tq, tk, tv, to, p, info.sm_count, st)
+                        : launch_prefill<64, 2>(tq, tk, tv, to, p, info.sm_count, st);
     if (cu_seqlens_k != nullptr)
-        return D == 128 ? launch_prefill<128, true>(tq, tk, tv, to, p, info.sm_count, st)
-                        : launch_prefill<64, true>(tq, tk, tv, to, p, info.sm_count, st);
-    return D == 128 ? launch_prefill<128, false>(tq, tk, tv, to, p, info.sm_count, st)
-                    : launch_prefill<64, false>(tq, tk, tv, to, p, info.sm_count, st);
+        return D == 128 ? launch_prefill<128, 1>(tq, tk, tv, to, p, info.sm_count, st)
+                        : launch_prefill<64, 1>(tq, tk, tv, to, p, info.sm_count, st);
+    return D == 128 ? launch_prefill<128, 0>(tq, tk, tv, to, p, info.sm_count, st)
+                    : launch_prefill<64, 0>(tq, tk, tv, to, p, info.sm_count, st);
 }
 
 }  // namespace swaa
@@ -381,6 +400,23 @@ extern "C" int swaa_prefill_chunked(const void* q, const void* k, const void* v,
     if (!cu_seqlens_k) return SWAA_ERR_INVALID_ARG;
     return prefill_impl(q, k, v, out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq, Hkv, D,
                         window, n_sink, is_full, scale, lse, stream);
+}
+
+extern "C" int swaa_prefill_paged(const void* q, const void* kpages, const void* vpages, void* out,
+                                  const int32_t* cu_seqlens_q, const int32_t* seqlens_k, const int32_t* block_table, int B,
+                                  int Tq, int max_seqlen_q, int max_blocks, int num_pages, int page_size, int Hq, int Hkv,
+                                  int D, int window, int n_sink, int is_full, float scale, float* lse, void* stream) {
+    if (!seqlens_k || !block_table) return SWAA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(block_table) & 3u) != 0) return SWAA_ERR_INVALID_ARG;
+    if (max_blocks < 1 || num_pages < 1 || page_size < 1) return SWAA_ERR_INVALID_ARG;
+    if (page_size % kPrefillBN != 0 || (long long)max_blocks * page_size > 2147483647LL) return SWAA_ERR_UNSUPPORTED;
+    PagedKV pg;
+    pg.block_table = block_table;
+    pg.max_blocks = max_blocks;
+    pg.num_pages = num_pages;
+    pg.page_size = page_size;
+    return prefill_impl(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, B, Tq, 0, max_seqlen_q, max_blocks * page_size, Hq,
+                        Hkv, D, window, n_sink, is_full, scale, lse, stream, pg);
 }
 
 // ------------------------------------------------------------------------------------ lazy ratio

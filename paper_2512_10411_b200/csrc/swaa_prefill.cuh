@@ -44,6 +44,10 @@ struct PrefillParams {
     const int32_t* cu_seqlens_k;  // nullable: keys of a chunked prefill, len_k >= len_q per sequence
     int B, T, max_seqlen, Hq, Hkv, G;
     int Tk, max_seqlen_k;         // packed key tokens and longest key sequence (chunked prefill only)
+    // paged keys/values (kMode 2): cu_seqlens_k holds the key LENGTHS [B]; entry j of sequence b lives in page
+    // block_table[b * max_blocks + j / page_size] at row j % page_size
+    const int32_t* block_table;
+    int max_blocks, page_size, num_pages;
     int pairs_per_kv;       // ceil(G / 2)
     int n_pairs;            // Hkv * pairs_per_kv
     int tiles_ub;           // upper bound on the number of query tiles over all sequences
@@ -226,7 +230,7 @@ struct PrefillSmem {
     static constexpr int kOffBar = kOffStage + 8 * 4096;
     // barriers: Q full/empty, K full/empty, V full/empty per stage, per side S-full / P-ready / O-done /
     // O-free, work-descriptor full/empty per slot, final
-    static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1;
+    static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1 + 1;
     static constexpr int kOffMisc = kOffBar + kNumBars * 8;      // tmem slot, abort flag, work descriptors
     static constexpr int kBytes = kOffMisc + 128;
     static constexpr int kDynamicBytes = kBytes + 1024;          // room to align the base to 1024 B
@@ -235,18 +239,20 @@ struct PrefillSmem {
 // One unit of work: a 128-row query tile of one sequence for one pair of query heads.
 struct WorkItem {
     int valid, seq_start, seq_len, m_tile, pair;
-    int k_start;  // first packed key token of the sequence (= seq_start for self attention)
+    int k_start;  // first packed key token of the sequence (= seq_start for self attention; sequence index when paged)
     int k_off;    // position of the sequence's first query inside its sequence: len_k - len_q (0 for self attention)
 };
 
-// kChunked: queries are the last len_q tokens of a longer key sequence (separate packing of the keys).
+// kMode 0: self attention.  1: chunked prefill, the queries are the last len_q tokens of a longer key sequence
+// (separate packing of the keys).  2: the same with keys and values in pages addressed through a block table.
 // The self-attention instance compiles the offsets away.
-template <int D, bool kChunked>
+template <int D, int kMode>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                const PrefillParams p) {
     using L = PrefillSmem<D>;
+    constexpr bool kChunked = kMode >= 1, kPaged = kMode == 2;
     constexpr int BM = kPrefillBM, BN = kPrefillBN;
     constexpr int ST = L::kStages;
     constexpr uint32_t kIdescQK = make_idesc(BM, BN, 0);
@@ -263,7 +269,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     constexpr int BAR_QF = 0, BAR_QE = 1, BAR_KF = 2, BAR_KE = BAR_KF + ST, BAR_VF = BAR_KE + ST, BAR_VE = BAR_VF + ST;
     constexpr int BAR_SF = BAR_VE + ST, BAR_PR = BAR_SF + 2, BAR_OD = BAR_PR + 2, BAR_OF = BAR_OD + 2;
     constexpr int BAR_WF = BAR_OF + 2, BAR_WE = BAR_WF + 2, BAR_FIN = BAR_WE + 2;
-    static_assert(BAR_FIN + 1 == L::kNumBars, "barrier count");
+    constexpr int BAR_VC = BAR_FIN + 1;  // paged only: the rows of a V tile past the last key have been cleared
+    static_assert(BAR_VC + 1 == L::kNumBars, "barrier count");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + L::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* work_ring = reinterpret_cast<volatile int*>(tmem_slot + 4);  // 2 slots x 8 ints
@@ -331,7 +338,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                     cur_ks = s0;
                     cur_off = 0;
-                    if (kChunked) {  // chunked prefill: the queries are the last `len` tokens
+                    if (kPaged) {  // keys in pages: cu_seqlens_k holds the key lengths
+                        const int lk = p.cu_seqlens_k[b];
+                        if (lk < len || lk > p.max_seqlen_k) {
+                            record_device_error(SWAA_ERR_BAD_SEQLENS);
+                            len = 0;
+                        }
+                        cur_ks = b;
+                        cur_off = lk - len;
+                    } else if (kChunked) {  // chunked prefill: the queries are the last `len` tokens
                         const int ks = p.cu_seqlens_k[b], ke = p.cu_seqlens_k[b + 1];
                         if (ke - ks < len || ke - ks > p.max_seqlen_k || ks < 0 || ke > p.Tk) {
                             record_device_error(SWAA_ERR_BAD_SEQLENS);
@@ -400,13 +415,24 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 for (int n = 0; n < nt; ++n, ++g) {
                     const int s = g % ST;
                     const uint32_t ph = (uint32_t)(g / ST) & 1u;
-                    const int tk = w.k_start + tr.tile(n) * BN;
+                    const int kt = tr.tile(n) * BN;  // first key of the tile, counted inside the sequence
+                    int tk = w.k_start + kt, page = 0;  // packed token index, or (row in page, page) when paged
+                    if (kPaged) {
+                        page = __ldg(p.block_table + (size_t)w.k_start * p.max_blocks + kt / p.page_size);
+                        tk = kt % p.page_size;
+                        if (page < 0 || page >= p.num_pages) {
+                            record_device_error(SWAA_ERR_BAD_SEQLENS);
+                            page = p.num_pages;  // out of range: the copy delivers zeros
+                        }
+                    }
                     ok = mbar_wait(bar(BAR_KE + s), ph ^ 1u, abort_flag);
                     if (!ok) break;
                     mbar_arrive_expect_tx(bar(BAR_KF + s), (uint32_t)L::kTileBytes);
 #pragma unroll
-                    for (int pn = 0; pn < L::kPanels; ++pn)
-                        tma_load_3d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, bar(BAR_KF + s));
+                    for (int pn = 0; pn < L::kPanels; ++pn) {
+                        if (kPaged) tma_load_4d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, page, bar(BAR_KF + s));
+                        else tma_load_3d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, bar(BAR_KF + s));
+                    }
                     ok = mbar_wait(bar(BAR_VE + s), ph ^ 1u, abort_flag);
                     if (!ok) {
                         mbar_wait(bar(BAR_KF + s), ph, abort_flag);  // the K copy just issued
@@ -414,8 +440,28 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                     mbar_arrive_expect_tx(bar(BAR_VF + s), (uint32_t)L::kTileBytes);
 #pragma unroll
-                    for (int pn = 0; pn < L::kPanels; ++pn)
-                        tma_load_3d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, bar(BAR_VF + s));
+                    for (int pn = 0; pn < L::kPanels; ++pn) {
+                        if (kPaged) tma_load_4d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, page, bar(BAR_VF + s));
+                        else tma_load_3d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, bar(BAR_VF + s));
+                    }
+                    if (kPaged) {
+                        // The rows of a page past the sequence's last key may hold anything (also NaN, and 0 * NaN is
+                        // NaN in the PV product): clear them in the V tile before the issuer may use it.  Only the last
+                        // key tile of a sequence that does not end on a tile boundary is concerned.
+                        const int first_bad = w.k_off + w.seq_len - kt;  // rows [first_bad, BN) lie past the last key
+                        if (first_bad < BN) {
+                            ok = mbar_wait(bar(BAR_VF + s), ph, abort_flag);
+                            if (!ok) break;
+                            for (int r = max(first_bad, 0); r < BN; ++r)
+#pragma unroll
+                                for (int pn = 0; pn < L::kPanels; ++pn)
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j)
+                                        st_shared_v4(sV + s * L::kTileBytes + pn * L::kPanelBytes + r * 128 + j * 16, 0u, 0u, 0u, 0u);
+                            fence_proxy_async_smem();
+                            mbar_arrive(bar(BAR_VC));
+                        }
+                    }
                 }
             }
             if (!ok) {
@@ -476,6 +522,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             int gs[2] = {0, 0};        // tiles processed per side (phase of S-full / P-ready / O-done)
             int items_side[2] = {0, 0};
             int items = 0;
+            int n_cleared = 0;  // V tiles whose rows past the sequence end were cleared (paged only)
             bool ok = true;
             for (int it = 0; ok; ++it) {
                 WorkItem w;
@@ -485,7 +532,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
                 const bool hasB = (hA + 1) < (hk + 1) * p.G;
                 const int i0 = w.m_tile * BM, i1 = min(w.seq_len, i0 + BM) - 1;
-                const int nt = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, p.n_sink, full).count();
+                const TileRange trng = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, p.n_sink, full);
+                const int nt = trng.count();
                 ok = mbar_wait(bar(BAR_QF), (uint32_t)items & 1u, abort_flag) &&
                      mbar_wait(bar(BAR_KF + g % ST), (uint32_t)(g / ST) & 1u, abort_flag);
                 if (!ok) break;
@@ -506,6 +554,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const uint32_t pk = (uint32_t)((g + 1) / ST) & 1u;
                     ok = mbar_wait(bar(BAR_PR + 0), (uint32_t)gs[0] & 1u, abort_flag) &&
                          mbar_wait(bar(BAR_VF + sv), pv, abort_flag);
+                    if (kPaged && ok && w.k_off + w.seq_len - trng.tile(n) * BN < BN) {
+                        // last key tile of a sequence that ends inside it: the producer clears the rows past the end
+                        ok = mbar_wait(bar(BAR_VC), (uint32_t)n_cleared & 1u, abort_flag);
+                        ++n_cleared;
+                    }
                     // the first PV of an item overwrites O: the previous item's epilogue must have read it
                     if (ok && n == 0) ok = mbar_wait(bar(BAR_OF + 0), ((uint32_t)items_side[0] & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
