@@ -468,6 +468,35 @@ def run_sweep():
     time_case("cfg2_full_causal", inputs.cfg_long(is_full=True), True, reps=3)
     time_case("cfg5_varlen", inputs.cfg_varlen(), False, reps=3)
     time_case("cfg1_tiny", inputs.cfg_tiny(), False)
+    # backward pass on workload 2 (five tile products per visible pair: 10 * D * Hq * pairs FLOP)
+    bcfg = inputs.cfg_long()
+    bq, bk, bv, bcu = inputs.make_prefill_inputs(bcfg, "cuda")
+    bT, bHq, bD = bq.shape
+    bout, bdo = torch.empty_like(bq), torch.randn(bq.shape, device="cuda").to(torch.bfloat16)
+    blse = torch.empty((bHq, bT), dtype=torch.float32, device="cuda")
+    swaa.swaa_prefill(bq, bk, bv, bout, bcu, bcfg.seqlens[0], bcfg.window, bcfg.n_sink, False, lse=blse)
+    bdq, bdk, bdv = torch.empty_like(bq), torch.empty_like(bk), torch.empty_like(bv)
+    bws = torch.empty(swaa.prefill_backward_workspace_size(bT, bHq, bD), dtype=torch.uint8, device="cuda")
+    ms = []
+    for r in range(4):
+        flush.zero_()
+        flush_rd.sum()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        swaa.swaa_prefill_backward(bq, bk, bv, bout, bdo, blse, bcu, bcfg.seqlens[0], bcfg.window, bcfg.n_sink, False, bdq,
+                                   bdk, bdv, bws)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if r > 0:
+            ms.append(a.elapsed_time(b))
+    assert swaa.last_device_status() == 0
+    ms.sort()
+    bflops = 10.0 * bD * bHq * visible_pairs(bcfg.seqlens[0], bcfg.window, bcfg.n_sink, False)
+    tf = bflops / (ms[len(ms) // 2] * 1e-3) / 1e12
+    print(json.dumps({"case": "backward_cfg2", "L": bcfg.seqlens[0], "Hq": bHq, "Hkv": bcfg.Hkv, "D": bD,
+                      "window": bcfg.window, "n_sink": bcfg.n_sink, "ms": ms[len(ms) // 2], "effective_tflops": tf,
+                      "frac_of_measured_peak": tf / peaks["bf16_tflops"]}), flush=True)
+    del bq, bk, bv, bout, bdo, bdq, bdk, bdv, bws
     # chunked prefill: a 4096-token chunk at the end of a 131072-token context (heads and mask of workload 2)
     g = torch.Generator(device="cuda").manual_seed(7)
     lq, lk, Hq, Hkv, D, W, S = 4096, 131072, 32, 8, 128, 2048, 4

@@ -93,6 +93,27 @@ int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out,
                          void* stream);
 
 /*
+ * Backward pass of swaa_prefill under the same mask policy (Sec. 3.3: fine-tuning under SWA uses the mask
+ * the model will be served with).  Given the forward inputs, the forward output `out`, its log-sum-exp
+ * rows `lse` (as written by swaa_prefill) and the gradient `dout` of the loss with respect to `out`, writes
+ * the gradients with respect to q, k and v (dk, dv summed over the query heads of each GQA group).
+ * Work is O(L * window) per head like the forward pass: a key tile only meets the query tiles that see it.
+ *
+ *   q, out, dout, dq  device, [T, Hq, D] bf16;  k, v, dk, dv  device, [T, Hkv, D] bf16
+ *   lse               device, float32 [Hq, T]
+ *   workspace         device, at least swaa_prefill_backward_workspace_size(T, Hq, D) bytes, 256-byte aligned;
+ *                     contents need not be initialised (an fp32 dq accumulator and the row terms dout.out)
+ * Other arguments and status codes as for swaa_prefill.  fp32 accumulation throughout; P and dS are rounded to
+ * bf16 for the tensor-core products, as in the forward pass.
+ */
+size_t swaa_prefill_backward_workspace_size(int T, int Hq, int D);
+
+int swaa_prefill_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
+                          const float* lse, const int32_t* cu_seqlens, int B, int T, int max_seqlen, int Hq, int Hkv,
+                          int D, int window, int n_sink, int is_full, float scale, void* dq, void* dk, void* dv,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Chunked prefill against a paged KV cache (the two needs of a serving engine that mixes prefill chunks and
  * decode steps, Sec. 4.1.1): queries as in swaa_prefill_chunked, keys and values as in swaa_decode_paged.
  *

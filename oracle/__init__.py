@@ -14,6 +14,8 @@ from .swaa_oracle import (  # noqa: F401
     lazy_ratio,
     num_threads,
     prefill,
+    prefill_backward,
+    prefill_backward_c,
     prefill_chunked,
     prefill_paged,
     visible,

@@ -238,6 +238,124 @@ int swaa_oracle_decode(const float* q, const float* kcache, const float* vcache,
 }
 
 /*
+ * Gradients of the packed self-attention prefill with respect to q, k, v for an upstream gradient dout
+ * (Sec. 3.3: fine-tuning under the SWA mask).  From out_i = sum_j p_ij v_j, p = softmax over the visible keys
+ * of s_ij = scale * q_i.k_j:
+ *     dv_j += p_ij dout_i;   dp_ij = dout_i . v_j;   ds_ij = p_ij (dp_ij - sum_j' p_ij' dp_ij');
+ *     dq_i = scale * sum_j ds_ij k_j;   dk_j += scale * ds_ij q_i     (dk, dv summed over the heads of a group).
+ * Two plain passes: rows (softmax statistics and dq), then keys (dk, dv from the rows that see them).
+ *   q, dout [T, Hq, D]; k, v [T, Hkv, D] float32 (bf16 values); dq [T, Hq, D], dk, dv [T, Hkv, D] double.
+ * Returns 0, or -1 on inconsistent arguments.
+ */
+int swaa_oracle_prefill_backward(const float* q, const float* k, const float* v, const float* dout,
+                                 const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D, int64_t W, int64_t S,
+                                 int is_full, double scale, double* dq, double* dk, double* dv) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
+    if (!is_full && W < 1) return -1;
+    if (S < 0) return -1;
+    const int G = Hq / Hkv;
+    const int64_t T = B > 0 ? cu_seqlens[B] : 0;
+    int64_t max_len = 0;
+    for (int b = 0; b < B; ++b) {
+        int64_t len = (int64_t)cu_seqlens[b + 1] - cu_seqlens[b];
+        if (len < 0) return -1;
+        if (len > max_len) max_len = len;
+    }
+    /* per (token, head): row maximum m, denominator den, and sum_j p_ij dp_ij */
+    double* rm = (double*)malloc(sizeof(double) * (size_t)(T * Hq > 0 ? T * Hq : 1));
+    double* rden = (double*)malloc(sizeof(double) * (size_t)(T * Hq > 0 ? T * Hq : 1));
+    double* rdot = (double*)malloc(sizeof(double) * (size_t)(T * Hq > 0 ? T * Hq : 1));
+#pragma omp parallel
+    {
+        double* sc = (double*)malloc(sizeof(double) * (size_t)(max_len > 0 ? max_len : 1));
+        double* dp = (double*)malloc(sizeof(double) * (size_t)(max_len > 0 ? max_len : 1));
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t r = 0; r < T * Hq; ++r) {
+            const int64_t t = r / Hq;
+            const int h = (int)(r % Hq), hk = h / G;
+            int b = 0;
+            while (!(cu_seqlens[b] <= t && t < cu_seqlens[b + 1])) ++b;
+            const int64_t s0 = cu_seqlens[b], i = t - s0;
+            const float* qi = q + r * D;
+            const float* gi = dout + r * D;
+            double m = -INFINITY;
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                const float* kj = k + ((s0 + j) * Hkv + hk) * (int64_t)D;
+                const float* vj = v + ((s0 + j) * Hkv + hk) * (int64_t)D;
+                double s = 0.0, d = 0.0;
+                for (int c = 0; c < D; ++c) {
+                    s += (double)qi[c] * (double)kj[c];
+                    d += (double)gi[c] * (double)vj[c];
+                }
+                sc[j] = s * scale;
+                dp[j] = d;
+                if (sc[j] > m) m = sc[j];
+            }
+            double den = 0.0, dot = 0.0;
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                den += exp(sc[j] - m);
+            }
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                dot += exp(sc[j] - m) / den * dp[j];
+            }
+            rm[r] = m;
+            rden[r] = den;
+            rdot[r] = dot;
+            double* dqi = dq + r * D;
+            for (int c = 0; c < D; ++c) dqi[c] = 0.0;
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                const double ds = exp(sc[j] - m) / den * (dp[j] - dot);
+                const float* kj = k + ((s0 + j) * Hkv + hk) * (int64_t)D;
+                for (int c = 0; c < D; ++c) dqi[c] += scale * ds * (double)kj[c];
+            }
+        }
+        free(sc);
+        free(dp);
+        /* keys: every (token, kv head) collects from the rows and heads that see it */
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t r = 0; r < T * Hkv; ++r) {
+            const int64_t t = r / Hkv;
+            const int hk = (int)(r % Hkv);
+            int b = 0;
+            while (!(cu_seqlens[b] <= t && t < cu_seqlens[b + 1])) ++b;
+            const int64_t s0 = cu_seqlens[b], len = cu_seqlens[b + 1] - s0, j = t - s0;
+            const float* kj = k + r * D;
+            const float* vj = v + r * D;
+            double* dkj = dk + r * D;
+            double* dvj = dv + r * D;
+            for (int c = 0; c < D; ++c) dkj[c] = dvj[c] = 0.0;
+            for (int64_t i = j; i < len; ++i) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                for (int h = hk * G; h < (hk + 1) * G; ++h) {
+                    const int64_t ri = (s0 + i) * Hq + h;
+                    const float* qi = q + ri * D;
+                    const float* gi = dout + ri * D;
+                    double s = 0.0, d = 0.0;
+                    for (int c = 0; c < D; ++c) {
+                        s += (double)qi[c] * (double)kj[c];
+                        d += (double)gi[c] * (double)vj[c];
+                    }
+                    const double p = exp(s * scale - rm[ri]) / rden[ri];
+                    const double ds = p * (d - rdot[ri]);
+                    for (int c = 0; c < D; ++c) {
+                        dvj[c] += p * (double)gi[c];
+                        dkj[c] += scale * ds * (double)qi[c];
+                    }
+                }
+            }
+        }
+    }
+    free(rm);
+    free(rden);
+    free(rdot);
+    return 0;
+}
+
+/*
  * Layer schedule (Sec. 3.1.2 fixed-interval FA layers; Sec. 3.1.1 FA decode;
  * Table 1 columns "FA layers" and "FA decode").  Layers fa_start, fa_start +
  * fa_step, ... keep full attention (fa_step == 0: none).  phase 0 = prefill,

@@ -48,6 +48,9 @@ def _load():
         lib.swaa_oracle_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
                                                     i64, vp, vp, vp, vp, vp, vp]
         lib.swaa_oracle_prefill_chunked.restype = ctypes.c_int
+        lib.swaa_oracle_prefill_backward.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
+                                                     vp, vp, vp]
+        lib.swaa_oracle_prefill_backward.restype = ctypes.c_int
         lib.swaa_oracle_decode.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
                                            vp, vp, vp, vp]
         lib.swaa_oracle_decode.restype = ctypes.c_int
@@ -242,3 +245,55 @@ def prefill_paged(q, kpages, vpages, cu_seqlens_q, seqlens_k, block_table, windo
     cu_k = np.concatenate([[0], np.cumsum(lk)])
     return prefill_chunked(q, np.concatenate(ks), np.concatenate(vs), cu_seqlens_q, cu_k, window, n_sink, is_full, scale,
                            rows)
+
+
+def prefill_backward_c(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_full: bool, scale: float | None = None):
+    """The same gradients as prefill_backward from the plain-C loops of swaa_oracle.c (fast enough for the sizes of
+    the GPU parity tests).  Returns dq [T,Hq,D], dk, dv [T,Hkv,D] float64."""
+    q, k, v, dout = _f32(q), _f32(k), _f32(v), _f32(dout)
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    dq = np.empty((T, Hq, D), dtype=np.float64)
+    dk = np.empty((T, Hkv, D), dtype=np.float64)
+    dv = np.empty((T, Hkv, D), dtype=np.float64)
+    rc = _load().swaa_oracle_prefill_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(cu), cu.shape[0] - 1, Hq, Hkv, D,
+                                              int(window), int(n_sink), int(bool(is_full)), float(scale), _ptr(dq),
+                                              _ptr(dk), _ptr(dv))
+    if rc != 0:
+        raise ValueError("swaa_oracle_prefill_backward: inconsistent arguments")
+    return {"dq": dq, "dk": dk, "dv": dv}
+
+
+def prefill_backward(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_full: bool, scale: float | None = None):
+    """Gradients of the masked softmax attention with respect to q, k, v for an upstream gradient dout, written
+    out row by row from the calculus of out_i = sum_j p_ij v_j, p = softmax over the visible keys of scale*q.k:
+        dv_j += p_ij dout_i;  dp_ij = dout_i . v_j;  ds_ij = p_ij (dp_ij - sum_j' p_ij' dp_ij');
+        dq_i = scale * sum_j ds_ij k_j;  dk_j += scale * ds_ij q_i      (dk, dv summed over the heads of a group).
+    Plain float64 numpy; returns dq [T,Hq,D], dk, dv [T,Hkv,D]."""
+    q, k, v, dout = (np.asarray(a, dtype=np.float64) for a in (q, k, v, dout))
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    for b in range(cu.shape[0] - 1):
+        s0, n = int(cu[b]), int(cu[b + 1] - cu[b])
+        for i in range(n):
+            keys = np.array([j for j in range(i + 1) if visible(i, j, window, n_sink, is_full)], dtype=np.int64) + s0
+            for h in range(Hq):
+                hk = h // G
+                s = (k[keys, hk] @ q[s0 + i, h]) * scale
+                p = np.exp(s - s.max())
+                p /= p.sum()
+                g = dout[s0 + i, h]
+                dv[keys, hk] += np.outer(p, g)
+                dp = v[keys, hk] @ g
+                ds = p * (dp - (p * dp).sum())
+                dq[s0 + i, h] = scale * (ds @ k[keys, hk])
+                dk[keys, hk] += scale * np.outer(ds, q[s0 + i, h])
+    return {"dq": dq, "dk": dk, "dv": dv}

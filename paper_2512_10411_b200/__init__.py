@@ -26,6 +26,8 @@ from .binding import (  # noqa: F401
     DECODE_STATIC_SCRATCH_BYTES,
     swaa_lazy_ratio,
     swaa_prefill,
+    swaa_prefill_backward,
+    prefill_backward_workspace_size,
     swaa_prefill_chunked,
     swaa_prefill_paged,
     last_device_status,

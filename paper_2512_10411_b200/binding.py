@@ -64,6 +64,10 @@ def load_library():
     lib.swaa_prefill.restype = ci
     lib.swaa_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     lib.swaa_prefill_chunked.restype = ci
+    lib.swaa_prefill_backward_workspace_size.argtypes = [ci, ci, ci]
+    lib.swaa_prefill_backward_workspace_size.restype = ctypes.c_size_t
+    lib.swaa_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.swaa_prefill_backward.restype = ci
     lib.swaa_prefill_paged.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     lib.swaa_prefill_paged.restype = ci
     lib.swaa_lazy_ratio.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
@@ -167,6 +171,34 @@ def swaa_prefill_chunked(q, k, v, out, cu_seqlens_q, cu_seqlens_k, max_seqlen_q:
                                   float(scale), _dev_ptr(lse, torch.float32, "lse"), _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_prefill_chunked")
+
+
+def prefill_backward_workspace_size(T, Hq, D) -> int:
+    """Forwards to C swaa_prefill_backward_workspace_size (bytes)."""
+    return int(load_library().swaa_prefill_backward_workspace_size(int(T), int(Hq), int(D)))
+
+
+def swaa_prefill_backward(q, k, v, out, dout, lse, cu_seqlens, max_seqlen: int, window: int, n_sink: int, is_full: bool,
+                          dq, dk, dv, workspace, scale: float = 0.0, stream=None) -> None:
+    """Forwards to C swaa_prefill_backward.  q, out, dout, dq [T,Hq,D]; k, v, dk, dv [T,Hkv,D] bf16; lse f32 [Hq,T];
+    workspace uint8 of prefill_backward_workspace_size(T, Hq, D) bytes."""
+    lib = load_library()
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    for name, t, shp in (("k", k, (T, Hkv, D)), ("v", v, (T, Hkv, D)), ("out", out, (T, Hq, D)), ("dout", dout, (T, Hq, D)),
+                         ("dq", dq, (T, Hq, D)), ("dk", dk, (T, Hkv, D)), ("dv", dv, (T, Hkv, D)), ("lse", lse, (Hq, T))):
+        if tuple(t.shape) != shp:
+            raise ValueError(f"swaa_prefill_backward: {name} must be {shp}")
+    B = cu_seqlens.numel() - 1
+    bf = torch.bfloat16
+    rc = lib.swaa_prefill_backward(_dev_ptr(q, bf, "q"), _dev_ptr(k, bf, "k"), _dev_ptr(v, bf, "v"), _dev_ptr(out, bf, "out"),
+                                   _dev_ptr(dout, bf, "dout"), _dev_ptr(lse, torch.float32, "lse"),
+                                   _dev_ptr(cu_seqlens, torch.int32, "cu_seqlens"), B, T, int(max_seqlen), Hq, Hkv, D,
+                                   int(window), int(n_sink), int(bool(is_full)), float(scale), _dev_ptr(dq, bf, "dq"),
+                                   _dev_ptr(dk, bf, "dk"), _dev_ptr(dv, bf, "dv"),
+                                   _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_prefill_backward")
 
 
 def swaa_prefill_paged(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, block_table, max_seqlen_q: int, window: int,

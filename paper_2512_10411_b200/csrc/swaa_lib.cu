@@ -11,6 +11,7 @@
 #include "swaa_internal.cuh"
 #include "swaa_decode.cuh"
 #include "swaa_prefill.cuh"
+#include "swaa_backward.cuh"
 
 namespace swaa {
 
@@ -417,6 +418,91 @@ extern "C" int swaa_prefill_paged(const void* q, const void* kpages, const void*
     pg.page_size = page_size;
     return prefill_impl(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, B, Tq, 0, max_seqlen_q, max_blocks * page_size, Hq,
                         Hkv, D, window, n_sink, is_full, scale, lse, stream, pg);
+}
+
+// -------------------------------------------------------------------------------------- backward
+namespace swaa {
+
+static size_t backward_workspace_bytes(int T, int Hq, int D, size_t* off_delta) {
+    const size_t acc = ((size_t)T * Hq * D * sizeof(float) + 255) / 256 * 256;
+    if (off_delta) *off_delta = acc;
+    return acc + (size_t)Hq * T * sizeof(float);
+}
+
+template <int D>
+static int launch_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
+                           const BackwardParams& p, void* dq, int max_seqlen, cudaStream_t st) {
+    using L = BackwardSmem<D>;
+    CUtensorMap tq, tk, tv, tdo;
+    int rc;
+    if ((rc = make_token_major_map(&tq, q, p.T, p.Hq, D, kBwdTile)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tk, k, p.T, p.Hkv, D, kBwdTile)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tv, v, p.T, p.Hkv, D, kBwdTile)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tdo, dout, p.T, p.Hq, D, kBwdTile)) != SWAA_OK) return rc;
+    const size_t n_acc = (size_t)p.T * p.Hq * D;
+    if (cudaMemsetAsync(p.dq_accum, 0, n_acc * sizeof(float), st) != cudaSuccess) return SWAA_ERR_CUDA;
+    const int rows = p.T * p.Hq;
+    backward_delta_kernel<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(dout), const_cast<float*>(p.delta), p.T,
+        p.Hq);
+    if (cudaFuncSetAttribute(backward_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
+        cudaSuccess)
+        return SWAA_ERR_CUDA;
+    const dim3 grid((unsigned)((max_seqlen + kBwdTile - 1) / kBwdTile), (unsigned)p.Hkv, (unsigned)p.B);
+    backward_kernel<D><<<grid, kBwdThreads, L::kDynamicBytes, st>>>(tq, tk, tv, tdo, p);
+    backward_convert_dq_kernel<<<(unsigned)((n_acc / 4 + 255) / 256 + 1), 256, 0, st>>>(
+        p.dq_accum, static_cast<__nv_bfloat16*>(dq), n_acc);
+    launch_counter().fetch_add(3, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
+}  // namespace swaa
+
+extern "C" size_t swaa_prefill_backward_workspace_size(int T, int Hq, int D) {
+    if (T < 1 || Hq < 1 || D < 1) return 256;
+    return backward_workspace_bytes(T, Hq, D, nullptr);
+}
+
+extern "C" int swaa_prefill_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
+                                     const float* lse, const int32_t* cu_seqlens, int B, int T, int max_seqlen, int Hq,
+                                     int Hkv, int D, int window, int n_sink, int is_full, float scale, void* dq, void* dk,
+                                     void* dv, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 0 || T < 0 || max_seqlen < 0 || Hq < 1 || Hkv < 1 || n_sink < 0) return SWAA_ERR_INVALID_ARG;
+    if (!is_full && window < 1) return SWAA_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0 || (D != 64 && D != 128)) return SWAA_ERR_UNSUPPORTED;
+    if (B > 65535 || Hkv > 65535) return SWAA_ERR_UNSUPPORTED;  // grid dimensions
+    if (B == 0 || T == 0 || max_seqlen == 0) return SWAA_OK;
+    if (!q || !k || !v || !out || !dout || !lse || !cu_seqlens || !dq || !dk || !dv) return SWAA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dout) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
+        return SWAA_ERR_INVALID_ARG;
+    size_t off_delta = 0;
+    const size_t need = backward_workspace_bytes(T, Hq, D, &off_delta);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < need)
+        return SWAA_ERR_WORKSPACE;
+    DeviceInfo info;
+    const int rc = current_device_info(&info);
+    if (rc != SWAA_OK) return rc;
+    if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
+    BackwardParams p;
+    p.lse = lse;
+    p.dq_accum = static_cast<float*>(workspace);
+    p.delta = reinterpret_cast<float*>(static_cast<char*>(workspace) + off_delta);
+    p.dk = static_cast<__nv_bfloat16*>(dk);
+    p.dv = static_cast<__nv_bfloat16*>(dv);
+    p.cu_seqlens = cu_seqlens;
+    p.B = B;
+    p.T = T;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.G = Hq / Hkv;
+    p.window = window;
+    p.n_sink = n_sink;
+    p.is_full = is_full ? 1 : 0;
+    p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return D == 128 ? launch_backward<128>(q, k, v, out, dout, p, dq, max_seqlen, st)
+                    : launch_backward<64>(q, k, v, out, dout, p, dq, max_seqlen, st);
 }
 
 // ------------------------------------------------------------------------------------ lazy ratio

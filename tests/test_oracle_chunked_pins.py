@@ -161,3 +161,31 @@ def test_lazy_ratio_equals_mass_from_two_log_sum_exps():
     a = oracle.prefill_chunked(q, k, v, cq, ck, recent, S, False)["lse"]
     b = oracle.prefill_chunked(q, k, v, cq, ck, 1, 0, True)["lse"]
     assert np.allclose(oracle.lazy_ratio(q, k, v, cq, ck, recent, S), np.exp(a - b).mean(axis=0), atol=1e-12)
+
+
+@pytest.mark.parametrize("W,S,full", [(5, 0, False), (4, 2, False), (1, 0, True), (100, 0, False)])
+def test_backward_matches_autograd_of_a_dense_masked_attention(W, S, full):
+    """The analytic gradients against torch.autograd (float64) through a dense masked softmax attention built
+    from a boolean mask matrix: a library routine the oracle's row formulas do not share anything with."""
+    lens, Hq, Hkv, D, scale = [9, 14], 4, 2, 8, 0.37
+    T = sum(lens)
+    q, k, v = _bf16_randn((T, Hq, D), 70), _bf16_randn((T, Hkv, D), 71), _bf16_randn((T, Hkv, D), 72)
+    dout = _bf16_randn((T, Hq, D), 73)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    got = oracle.prefill_backward(q, k, v, dout, cu, W, S, full, scale=scale)
+    tq, tk, tv = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (q, k, v))
+    outs = []
+    for b, n in enumerate(lens):
+        s0 = int(cu[b])
+        i, j = torch.arange(n)[:, None], torch.arange(n)[None, :]
+        mask = (j <= i) & (torch.tensor(full) | (j > i - W) | (j < S))
+        kk = tk[s0:s0 + n].repeat_interleave(Hq // Hkv, dim=1)
+        vv = tv[s0:s0 + n].repeat_interleave(Hq // Hkv, dim=1)
+        sc = torch.einsum("ihd,jhd->hij", tq[s0:s0 + n], kk) * scale
+        sc = sc.masked_fill(~mask[None], float("-inf"))
+        outs.append(torch.einsum("hij,jhd->ihd", torch.softmax(sc, dim=-1), vv))
+    torch.cat(outs).backward(torch.tensor(dout, dtype=torch.float64))
+    fast = oracle.prefill_backward_c(q, k, v, dout, cu, W, S, full, scale=scale)
+    for name, t in (("dq", tq), ("dk", tk), ("dv", tv)):
+        assert np.allclose(got[name], t.grad.numpy(), rtol=0, atol=1e-11), name
+        assert np.allclose(fast[name], t.grad.numpy(), rtol=0, atol=1e-11), name + " (C loops)"
