@@ -476,7 +476,7 @@ def run_sweep():
     blse = torch.empty((bHq, bT), dtype=torch.float32, device="cuda")
     swaa.swaa_prefill(bq, bk, bv, bout, bcu, bcfg.seqlens[0], bcfg.window, bcfg.n_sink, False, lse=blse)
     bdq, bdk, bdv = torch.empty_like(bq), torch.empty_like(bk), torch.empty_like(bv)
-    bws = torch.empty(swaa.prefill_backward_workspace_size(bT, bHq, bD), dtype=torch.uint8, device="cuda")
+    bws = torch.empty(swaa.prefill_backward_workspace_size(1, bT, bHq, bcfg.Hkv, bD, bcfg.n_sink), dtype=torch.uint8, device="cuda")
     ms = []
     for r in range(4):
         flush.zero_()

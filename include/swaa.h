@@ -101,12 +101,13 @@ int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out,
  *
  *   q, out, dout, dq  device, [T, Hq, D] bf16;  k, v, dk, dv  device, [T, Hkv, D] bf16
  *   lse               device, float32 [Hq, T]
- *   workspace         device, at least swaa_prefill_backward_workspace_size(T, Hq, D) bytes, 256-byte aligned;
- *                     contents need not be initialised (an fp32 dq accumulator and the row terms dout.out)
+ *   workspace         device, at least swaa_prefill_backward_workspace_size(B, T, Hq, Hkv, D, n_sink) bytes,
+ *                     256-byte aligned; contents need not be initialised (fp32 accumulators for dq and for the
+ *                     dk, dv rows of the sink key tiles, and the row terms dout.out and lse * log2(e))
  * Other arguments and status codes as for swaa_prefill.  fp32 accumulation throughout; P and dS are rounded to
  * bf16 for the tensor-core products, as in the forward pass.
  */
-size_t swaa_prefill_backward_workspace_size(int T, int Hq, int D);
+size_t swaa_prefill_backward_workspace_size(int B, int T, int Hq, int Hkv, int D, int n_sink);
 
 int swaa_prefill_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
                           const float* lse, const int32_t* cu_seqlens, int B, int T, int max_seqlen, int Hq, int Hkv,

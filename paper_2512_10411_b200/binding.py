@@ -64,7 +64,7 @@ def load_library():
     lib.swaa_prefill.restype = ci
     lib.swaa_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     lib.swaa_prefill_chunked.restype = ci
-    lib.swaa_prefill_backward_workspace_size.argtypes = [ci, ci, ci]
+    lib.swaa_prefill_backward_workspace_size.argtypes = [ci, ci, ci, ci, ci, ci]
     lib.swaa_prefill_backward_workspace_size.restype = ctypes.c_size_t
     lib.swaa_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.swaa_prefill_backward.restype = ci
@@ -173,15 +173,15 @@ def swaa_prefill_chunked(q, k, v, out, cu_seqlens_q, cu_seqlens_k, max_seqlen_q:
         raise SwaaError(rc, "swaa_prefill_chunked")
 
 
-def prefill_backward_workspace_size(T, Hq, D) -> int:
+def prefill_backward_workspace_size(B, T, Hq, Hkv, D, n_sink) -> int:
     """Forwards to C swaa_prefill_backward_workspace_size (bytes)."""
-    return int(load_library().swaa_prefill_backward_workspace_size(int(T), int(Hq), int(D)))
+    return int(load_library().swaa_prefill_backward_workspace_size(int(B), int(T), int(Hq), int(Hkv), int(D), int(n_sink)))
 
 
 def swaa_prefill_backward(q, k, v, out, dout, lse, cu_seqlens, max_seqlen: int, window: int, n_sink: int, is_full: bool,
                           dq, dk, dv, workspace, scale: float = 0.0, stream=None) -> None:
     """Forwards to C swaa_prefill_backward.  q, out, dout, dq [T,Hq,D]; k, v, dk, dv [T,Hkv,D] bf16; lse f32 [Hq,T];
-    workspace uint8 of prefill_backward_workspace_size(T, Hq, D) bytes."""
+    workspace uint8 of prefill_backward_workspace_size(B, T, Hq, Hkv, D, n_sink) bytes."""
     lib = load_library()
     T, Hq, D = q.shape
     Hkv = k.shape[1]

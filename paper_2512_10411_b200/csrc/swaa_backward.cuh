@@ -27,8 +27,12 @@
 namespace swaa {
 
 struct BackwardParams {
-    const float* lse;        // [Hq, T] natural log
+    const float* lse;        // [Hq, T] natural log (forward output)
+    const float* lse2;       // [Hq, T] the same times log2(e), written with delta
     const float* delta;      // [Hq, T]
+    float* dkv_accum;        // [2][B][sink_rows][Hkv][D] fp32, zeroed: dk, dv of the sink tiles, which are split over blocks
+    int sink_tiles;          // key tiles that hold sink keys (their query range is cut into chunks), 0 for full attention
+    int chunks;              // blocks per sink tile
     float* dq_accum;         // [T, Hq, D] fp32, zeroed before the launch
     __nv_bfloat16* dk;       // [T, Hkv, D]
     __nv_bfloat16* dv;
@@ -40,24 +44,27 @@ struct BackwardParams {
 
 constexpr int kBwdTile = 64;      // keys per block and query rows per step
 constexpr int kBwdThreads = 128;  // four warps, 16 keys each
+constexpr int kBwdChunkTiles = 32; // query tiles per block of a sink key tile
 
 template <int D>
 struct BackwardSmem {
     static constexpr int kPanels = D / 64;
     static constexpr int kPanelBytes = kBwdTile * 128;
     static constexpr int kTileBytes = kPanels * kPanelBytes;  // one [64][D] bf16 tile
-    static constexpr int kOffK = 0, kOffV = kTileBytes, kOffQ = 2 * kTileBytes, kOffDO = 3 * kTileBytes;
-    static constexpr int kOffDS = 4 * kTileBytes;             // dS^T [64 keys][64 rows] bf16, 128-byte rows, swizzled
-    static constexpr int kOffRow = kOffDS + kBwdTile * 128;   // lse, delta of the 64 rows (fp32)
-    static constexpr int kOffBar = kOffRow + 2 * kBwdTile * 4;
-    static constexpr int kBytes = kOffBar + 2 * 8 + 16;
+    static constexpr int kOffK = 0, kOffV = kTileBytes;
+    static constexpr int kOffQ = 2 * kTileBytes;              // two buffers of (Q tile, dO tile)
+    static constexpr int kOffDS = 6 * kTileBytes;             // dS^T [64 keys][64 rows] bf16, 128-byte rows, swizzled
+    static constexpr int kOffRow = kOffDS + kBwdTile * 128;   // two buffers of (lse * log2e, delta) of the 64 rows (fp32)
+    static constexpr int kOffBar = kOffRow + 4 * kBwdTile * 4;
+    static constexpr int kBytes = kOffBar + 3 * 8 + 16;
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
 
 // delta[h, t] = sum_d out[t, h, d] * dout[t, h, d]; one warp per (t, h).
 template <int D>
 __global__ void backward_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
-                                      float* __restrict__ delta, int T, int Hq) {
+                                      const float* __restrict__ lse, float* __restrict__ delta,
+                                      float* __restrict__ lse2, int T, int Hq) {
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (row >= T * Hq) return;
     const int t = row / Hq, h = row - t * Hq;
@@ -70,7 +77,10 @@ __global__ void backward_delta_kernel(const __nv_bfloat16* __restrict__ out, con
         acc += a.x * b.x + a.y * b.y;
     }
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    if (lane == 0) delta[(size_t)h * T + t] = acc;
+    if (lane == 0) {
+        delta[(size_t)h * T + t] = acc;
+        lse2[(size_t)h * T + t] = lse[(size_t)h * T + t] * 1.4426950408889634f;
+    }
 }
 
 // dq = bf16(dq_accum)
@@ -82,6 +92,24 @@ __global__ void backward_convert_dq_kernel(const float* __restrict__ acc, __nv_b
     } else {
         for (size_t j = i; j < n; ++j) dq[j] = __float2bfloat16_rn(acc[j]);
     }
+}
+
+// dk, dv rows of the split key tiles = bf16(dkv_accum); one thread per four channels of one (b, row, kv head).
+__global__ void backward_convert_dkv_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dk,
+                                            __nv_bfloat16* __restrict__ dv, const int32_t* __restrict__ cu_seqlens, int B,
+                                            int T, int sink_rows, int Hkv, int D) {
+    const size_t plane = (size_t)B * sink_rows * Hkv * D;
+    const size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (e >= plane) return;
+    const size_t row = e / ((size_t)Hkv * D);  // b * sink_rows + j
+    const int b = (int)(row / sink_rows), j = (int)(row - (size_t)b * sink_rows);
+    const int seq_start = cu_seqlens[b], Lseq = cu_seqlens[b + 1] - seq_start;
+    if (j >= Lseq || seq_start < 0 || seq_start + Lseq > T) return;
+    const size_t dst = (size_t)(seq_start + j) * Hkv * D + (e - row * (size_t)Hkv * D);
+    const float4 a = *reinterpret_cast<const float4*>(acc + e);
+    const float4 c = *reinterpret_cast<const float4*>(acc + plane + e);
+    *reinterpret_cast<uint2*>(dk + dst) = make_uint2(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w));
+    *reinterpret_cast<uint2*>(dv + dst) = make_uint2(pack_bf16x2(c.x, c.y), pack_bf16x2(c.z, c.w));
 }
 
 // Address of the 16-byte chunk `chunk` (0..D/8-1) of row `row` of a [64][D] tile stored as 64-channel
@@ -103,15 +131,23 @@ backward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t sK = smem_base + L::kOffK, sV = smem_base + L::kOffV, sQ = smem_base + L::kOffQ;
-    const uint32_t sDO = smem_base + L::kOffDO, sDS = smem_base + L::kOffDS;
-    float* s_lse = reinterpret_cast<float*>(smem_gen + L::kOffRow);
-    float* s_delta = s_lse + BT;
-    const uint32_t bar_kv = smem_base + L::kOffBar, bar_q = bar_kv + 8;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + L::kOffBar + 16);
+    const uint32_t sK = smem_base + L::kOffK, sV = smem_base + L::kOffV, sDS = smem_base + L::kOffDS;
+    const uint32_t sQD = smem_base + L::kOffQ;  // buffer u: Q at sQD + u * 2 * tile, dO one tile further
+    float* s_rows = reinterpret_cast<float*>(smem_gen + L::kOffRow);  // buffer u: lse2 at [u*128 .. +63], delta at [+64 ..]
+    const uint32_t bar_kv = smem_base + L::kOffBar, bar_q0 = bar_kv + 8;  // bar_q0 + 8 * u
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + L::kOffBar + 24);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
-    const int n_tile = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+    const int hk = blockIdx.y, b = blockIdx.z;
+    // blockIdx.x -> (key tile, chunk of its query range): the tiles that hold sink keys meet every later query
+    // tile, so their range is cut into chunks of kBwdChunkTiles query tiles handled by separate blocks
+    int n_tile, chunk = -1;
+    if ((int)blockIdx.x < p.sink_tiles * p.chunks) {
+        n_tile = (int)blockIdx.x / p.chunks;
+        chunk = (int)blockIdx.x - n_tile * p.chunks;
+    } else {
+        n_tile = p.sink_tiles + ((int)blockIdx.x - p.sink_tiles * p.chunks);
+    }
     const int seq_start = p.cu_seqlens[b], Lseq = p.cu_seqlens[b + 1] - seq_start;
     const int j0 = n_tile * BT;
     if (Lseq <= 0 || j0 >= Lseq || seq_start < 0 || seq_start + Lseq > p.T) {
@@ -121,17 +157,47 @@ backward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const bool full = p.is_full != 0;
     const int j1 = min(j0 + BT, Lseq) - 1;
     // query tiles that can see this key tile: the band above it; all later ones if it holds sink keys
-    const int m_lo = j0 / BT;
-    const int m_hi = (full || j0 < p.n_sink) ? (Lseq - 1) / BT
-                                             : (int)(min((long long)Lseq - 1, (long long)j1 + p.window - 1) / BT);
+    int m_lo = j0 / BT;
+    int m_hi = (full || j0 < p.n_sink) ? (Lseq - 1) / BT
+                                       : (int)(min((long long)Lseq - 1, (long long)j1 + p.window - 1) / BT);
+    const bool split = chunk >= 0;  // dK, dV of this tile come from several blocks: accumulate in fp32
+    if (split) {
+        m_lo += chunk * kBwdChunkTiles;
+        m_hi = min(m_hi, m_lo + kBwdChunkTiles - 1);
+        if (m_lo > m_hi) return;
+    }
+    const int nm = m_hi - m_lo + 1, n_steps = nm * p.G;
 
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar_kv, 1u);
-        mbar_init(bar_q, 1u);
+        mbar_init(bar_q0, 1u);
+        mbar_init(bar_q0 + 8, 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Loads of step s (query head hq = s / nm, query tile m = m_lo + s % nm) into buffer s & 1: Q and dO tiles by
+    // TMA, the 64 row terms by 4-byte asynchronous copies (zero-filled past the end of the sequence).
+    auto issue_step = [&](int s_) {
+        const int u = s_ & 1, h_ = hk * p.G + s_ / nm, i0_ = (m_lo + s_ % nm) * BT;
+        if (tid == 0) {
+            const uint32_t dst = sQD + (uint32_t)u * 2u * L::kTileBytes, bq = bar_q0 + 8u * (uint32_t)u;
+            mbar_arrive_expect_tx(bq, 2u * (uint32_t)L::kTileBytes);
+#pragma unroll
+            for (int pn = 0; pn < L::kPanels; ++pn) {
+                tma_load_3d(dst + pn * L::kPanelBytes, &tm_q, pn * 64, h_, seq_start + i0_, bq);
+                tma_load_3d(dst + L::kTileBytes + pn * L::kPanelBytes, &tm_do, pn * 64, h_, seq_start + i0_, bq);
+            }
+        }
+        {
+            const int r = tid & 63, i = i0_ + r;
+            const float* src = (tid < 64 ? p.lse2 : p.delta) + (size_t)h_ * p.T + seq_start + (i < Lseq ? i : 0);
+            const uint32_t dsts = smem_u32(s_rows + u * 128 + tid);
+            const int nbytes = i < Lseq ? 4 : 0;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dsts), "l"(src), "r"(nbytes) : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+    };
     if (tid == 0) {
         mbar_arrive_expect_tx(bar_kv, 2u * (uint32_t)L::kTileBytes);
 #pragma unroll
@@ -140,6 +206,7 @@ backward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tma_load_3d(sV + pn * L::kPanelBytes, &tm_v, pn * 64, hk, seq_start + j0, bar_kv);
         }
     }
+    issue_step(0);
     bool ok = __syncthreads_and(mbar_wait(bar_kv, 0u, abort_flag)) != 0;  // one decision for the whole block
 
     float dk_acc[ND][4], dv_acc[ND][4];
@@ -151,27 +218,19 @@ backward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const float sl2 = p.scale * 1.4426950408889634f;
     const int krow = 16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1);  // A fragments of K_w / V_w (non-transposed)
     const int kchk = lane >> 4;
-    uint32_t step = 0;
-    for (int hq = 0; hq < p.G && ok; ++hq) {
-        const int h = hk * p.G + hq;
-        for (int m = m_lo; m <= m_hi && ok; ++m, ++step) {
-            const int i0 = m * BT;
-            __syncthreads();  // everybody is done with the previous Q, dO, dS^T and row data
-            if (tid == 0) {
-                mbar_arrive_expect_tx(bar_q, 2u * (uint32_t)L::kTileBytes);
-#pragma unroll
-                for (int pn = 0; pn < L::kPanels; ++pn) {
-                    tma_load_3d(sQ + pn * L::kPanelBytes, &tm_q, pn * 64, h, seq_start + i0, bar_q);
-                    tma_load_3d(sDO + pn * L::kPanelBytes, &tm_do, pn * 64, h, seq_start + i0, bar_q);
-                }
-            }
-            if (tid < BT) {
-                const int i = i0 + tid;
-                s_lse[tid] = i < Lseq ? p.lse[(size_t)h * p.T + seq_start + i] * 1.4426950408889634f : 0.f;
-                s_delta[tid] = i < Lseq ? p.delta[(size_t)h * p.T + seq_start + i] : 0.f;
-            }
-            ok = __syncthreads_and(mbar_wait(bar_q, step & 1u, abort_flag)) != 0;  // also publishes the row data
+    for (int step = 0; step < n_steps && ok; ++step) {
+        {
+            const int u = step & 1;
+            const int h = hk * p.G + step / nm, i0 = (m_lo + step % nm) * BT;
+            const uint32_t sQ = sQD + (uint32_t)u * 2u * L::kTileBytes, sDO = sQ + L::kTileBytes;
+            const float* s_lse = s_rows + u * 128;
+            const float* s_delta = s_lse + 64;
+            // this step's tiles and row terms have landed; every warp is done with the previous step, whose
+            // buffers (and dS^T) may now be refilled
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            ok = __syncthreads_and(mbar_wait(bar_q0 + 8u * (uint32_t)u, (uint32_t)(step >> 1) & 1u, abort_flag)) != 0;
             if (!ok) break;
+            if (step + 1 < n_steps) issue_step(step + 1);
 
             // ---- S^T = K_w Q^T and dP^T = V_w dO^T : [16 keys] x [64 rows]
             float st[8][4], dpt[8][4];
@@ -277,6 +336,24 @@ backward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     if (!ok) return;
     // ---- dK, dV rows of this warp's keys
+    if (split) {
+        const int sink_rows = p.sink_tiles * BT;
+        const size_t plane = (size_t)p.B * sink_rows * p.Hkv * D;
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh) {
+            const int j = j0 + 16 * warp + g + 8 * kh;
+            if (j < Lseq) {
+                float* dkr = p.dkv_accum + (((size_t)b * sink_rows + j) * p.Hkv + hk) * D + 2 * c;
+#pragma unroll
+                for (int nd = 0; nd < ND; ++nd) {
+                    atomicAdd(reinterpret_cast<float2*>(dkr + 8 * nd), make_float2(dk_acc[nd][2 * kh], dk_acc[nd][2 * kh + 1]));
+                    atomicAdd(reinterpret_cast<float2*>(dkr + plane + 8 * nd),
+                              make_float2(dv_acc[nd][2 * kh], dv_acc[nd][2 * kh + 1]));
+                }
+            }
+        }
+        return;
+    }
 #pragma unroll
     for (int kh = 0; kh < 2; ++kh) {
         const int j = j0 + 16 * warp + g + 8 * kh;

@@ -423,15 +423,28 @@ extern "C" int swaa_prefill_paged(const void* q, const void* kpages, const void*
 // -------------------------------------------------------------------------------------- backward
 namespace swaa {
 
-static size_t backward_workspace_bytes(int T, int Hq, int D, size_t* off_delta) {
-    const size_t acc = ((size_t)T * Hq * D * sizeof(float) + 255) / 256 * 256;
-    if (off_delta) *off_delta = acc;
-    return acc + (size_t)Hq * T * sizeof(float);
+// Workspace: [dq accumulator | dk, dv accumulators of the split sink tiles] (zeroed by one memset) | delta | lse2.
+struct BackwardWorkspace {
+    size_t off_dkv, zero_bytes, off_delta, off_lse2, bytes;
+    int sink_rows;
+};
+
+static BackwardWorkspace backward_workspace(int B, int T, int Hq, int Hkv, int D, int n_sink) {
+    BackwardWorkspace w;
+    const long long t_rows = ((long long)T + kBwdTile - 1) / kBwdTile * kBwdTile;
+    const long long s_rows = ((long long)n_sink + kBwdTile - 1) / kBwdTile * kBwdTile;
+    w.sink_rows = (int)(s_rows < t_rows ? s_rows : t_rows);
+    w.off_dkv = ((size_t)T * Hq * D * sizeof(float) + 255) / 256 * 256;
+    w.zero_bytes = w.off_dkv + 2 * (size_t)B * w.sink_rows * Hkv * D * sizeof(float);
+    w.off_delta = (w.zero_bytes + 255) / 256 * 256;
+    w.off_lse2 = w.off_delta + ((size_t)Hq * T * sizeof(float) + 255) / 256 * 256;
+    w.bytes = w.off_lse2 + (size_t)Hq * T * sizeof(float);
+    return w;
 }
 
 template <int D>
 static int launch_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
-                           const BackwardParams& p, void* dq, int max_seqlen, cudaStream_t st) {
+                           const BackwardParams& p, void* dq, int max_seqlen, size_t zero_bytes, cudaStream_t st) {
     using L = BackwardSmem<D>;
     CUtensorMap tq, tk, tv, tdo;
     int rc;
@@ -440,27 +453,36 @@ static int launch_backward(const void* q, const void* k, const void* v, const vo
     if ((rc = make_token_major_map(&tv, v, p.T, p.Hkv, D, kBwdTile)) != SWAA_OK) return rc;
     if ((rc = make_token_major_map(&tdo, dout, p.T, p.Hq, D, kBwdTile)) != SWAA_OK) return rc;
     const size_t n_acc = (size_t)p.T * p.Hq * D;
-    if (cudaMemsetAsync(p.dq_accum, 0, n_acc * sizeof(float), st) != cudaSuccess) return SWAA_ERR_CUDA;
+    if (cudaMemsetAsync(p.dq_accum, 0, zero_bytes, st) != cudaSuccess) return SWAA_ERR_CUDA;
     const int rows = p.T * p.Hq;
     backward_delta_kernel<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(dout), const_cast<float*>(p.delta), p.T,
-        p.Hq);
+        static_cast<const __nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(dout), p.lse,
+        const_cast<float*>(p.delta), const_cast<float*>(p.lse2), p.T, p.Hq);
     if (cudaFuncSetAttribute(backward_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
         cudaSuccess)
         return SWAA_ERR_CUDA;
-    const dim3 grid((unsigned)((max_seqlen + kBwdTile - 1) / kBwdTile), (unsigned)p.Hkv, (unsigned)p.B);
+    const int ntiles = (max_seqlen + kBwdTile - 1) / kBwdTile;
+    const dim3 grid((unsigned)(p.sink_tiles * p.chunks + (ntiles - p.sink_tiles)), (unsigned)p.Hkv, (unsigned)p.B);
     backward_kernel<D><<<grid, kBwdThreads, L::kDynamicBytes, st>>>(tq, tk, tv, tdo, p);
     backward_convert_dq_kernel<<<(unsigned)((n_acc / 4 + 255) / 256 + 1), 256, 0, st>>>(
         p.dq_accum, static_cast<__nv_bfloat16*>(dq), n_acc);
-    launch_counter().fetch_add(3, std::memory_order_relaxed);
+    int launches = 3;
+    if (p.sink_tiles > 0) {
+        const int sink_rows = p.sink_tiles * kBwdTile;
+        const size_t plane = (size_t)p.B * sink_rows * p.Hkv * D;
+        backward_convert_dkv_kernel<<<(unsigned)((plane / 4 + 255) / 256), 256, 0, st>>>(
+            p.dkv_accum, p.dk, p.dv, p.cu_seqlens, p.B, p.T, sink_rows, p.Hkv, D);
+        ++launches;
+    }
+    launch_counter().fetch_add((uint64_t)launches, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
 }  // namespace swaa
 
-extern "C" size_t swaa_prefill_backward_workspace_size(int T, int Hq, int D) {
-    if (T < 1 || Hq < 1 || D < 1) return 256;
-    return backward_workspace_bytes(T, Hq, D, nullptr);
+extern "C" size_t swaa_prefill_backward_workspace_size(int B, int T, int Hq, int Hkv, int D, int n_sink) {
+    if (B < 1 || T < 1 || Hq < 1 || Hkv < 1 || D < 1 || n_sink < 0) return 256;
+    return backward_workspace(B, T, Hq, Hkv, D, n_sink).bytes;
 }
 
 extern "C" int swaa_prefill_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
@@ -476,18 +498,20 @@ extern "C" int swaa_prefill_backward(const void* q, const void* k, const void* v
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dout) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv))
         return SWAA_ERR_INVALID_ARG;
-    size_t off_delta = 0;
-    const size_t need = backward_workspace_bytes(T, Hq, D, &off_delta);
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < need)
+    const BackwardWorkspace w = backward_workspace(B, T, Hq, Hkv, D, n_sink);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < w.bytes)
         return SWAA_ERR_WORKSPACE;
     DeviceInfo info;
     const int rc = current_device_info(&info);
     if (rc != SWAA_OK) return rc;
     if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
+    char* ws = static_cast<char*>(workspace);
     BackwardParams p;
     p.lse = lse;
-    p.dq_accum = static_cast<float*>(workspace);
-    p.delta = reinterpret_cast<float*>(static_cast<char*>(workspace) + off_delta);
+    p.dq_accum = reinterpret_cast<float*>(ws);
+    p.dkv_accum = reinterpret_cast<float*>(ws + w.off_dkv);
+    p.delta = reinterpret_cast<float*>(ws + w.off_delta);
+    p.lse2 = reinterpret_cast<float*>(ws + w.off_lse2);
     p.dk = static_cast<__nv_bfloat16*>(dk);
     p.dv = static_cast<__nv_bfloat16*>(dv);
     p.cu_seqlens = cu_seqlens;
@@ -500,9 +524,23 @@ extern "C" int swaa_prefill_backward(const void* q, const void* k, const void* v
     p.n_sink = n_sink;
     p.is_full = is_full ? 1 : 0;
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
+    // Key tiles that hold sink keys meet every later query tile: with long sequences their query range is cut
+    // into chunks handled by separate blocks, which add dk, dv into the fp32 accumulators.
+    const int ntiles = (max_seqlen + kBwdTile - 1) / kBwdTile;
+    p.chunks = (ntiles + kBwdChunkTiles - 1) / kBwdChunkTiles;
+    p.sink_tiles = 0;
+    if (!is_full && p.chunks > 1) {
+        const int st_need = (int)(((long long)n_sink + kBwdTile - 1) / kBwdTile);
+        p.sink_tiles = st_need < ntiles ? st_need : ntiles;
+        if (p.sink_tiles * kBwdTile > w.sink_rows) p.sink_tiles = w.sink_rows / kBwdTile;
+    }
+    if (p.sink_tiles == 0) p.chunks = 1;
+    if ((long long)p.sink_tiles * p.chunks + (ntiles - p.sink_tiles) > 0x7fffffffLL) return SWAA_ERR_UNSUPPORTED;
+    const size_t zero_bytes = p.sink_tiles > 0 ? w.off_dkv + 2 * (size_t)B * p.sink_tiles * kBwdTile * Hkv * D * sizeof(float)
+                                               : (size_t)T * Hq * D * sizeof(float);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return D == 128 ? launch_backward<128>(q, k, v, out, dout, p, dq, max_seqlen, st)
-                    : launch_backward<64>(q, k, v, out, dout, p, dq, max_seqlen, st);
+    return D == 128 ? launch_backward<128>(q, k, v, out, dout, p, dq, max_seqlen, zero_bytes, st)
+                    : launch_backward<64>(q, k, v, out, dout, p, dq, max_seqlen, zero_bytes, st);
 }
 
 // ------------------------------------------------------------------------------------ lazy ratio

@@ -63,7 +63,7 @@ def run_forward_backward(cfg, scale=0.0):
     out = torch.empty_like(q)
     lse = torch.empty((Hq, T), dtype=torch.float32, device="cuda")
     swaa.swaa_prefill(q, k, v, out, cu, max(cfg.seqlens), cfg.window, cfg.n_sink, cfg.is_full, scale=scale, lse=lse)
-    nbytes = swaa.prefill_backward_workspace_size(T, Hq, D)
+    nbytes = swaa.prefill_backward_workspace_size(len(cfg.seqlens), T, Hq, cfg.Hkv, D, cfg.n_sink)
     guard = 4096
     ws_all = torch.full((nbytes + 2 * guard,), 0xA5, dtype=torch.uint8, device="cuda")
     ws = ws_all[guard:guard + nbytes]
