@@ -35,7 +35,7 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists).
-PREFILL_DRAM_TRAFFIC_BYTES = 643980800  # 405.03 MB read + 238.95 MB written, profiles/prefill_kernel_cfg2_long_swa.txt
+PREFILL_DRAM_TRAFFIC_BYTES = 639519488  # 404.52 MB read + 235.00 MB written, profiles/prefill_kernel_cfg2_long_swa.txt
 
 # decode kernel: 4 x (1.0739 GB read + 4 MB written) scaled from the B=4 capture; 270.0 MB + 5 MB at full size
 DECODE_FA_DRAM_TRAFFIC_BYTES = 4 * (1073919000 + 4249600)
@@ -362,7 +362,7 @@ def run_ours(args, rank, local_rank, world):
                 "h2d_bytes_per_step": int(q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": int(out.numel()) * 2,
                 "ms_per_step": e2e_ms},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "prefill_kernel<128, false>", "bound": "tensor", "achieved": achieved,
+        "roofline": {"kernel": "prefill_kernel<128, 0>", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                      "traffic": PREFILL_DRAM_TRAFFIC_BYTES, "peak_source": peaks["source"] + " burst bf16",
                      "frac_of_nominal_2250": achieved / 2250.0, "ms_per_launch": avg_pre_ms},

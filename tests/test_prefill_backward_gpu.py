@@ -117,3 +117,10 @@ def test_backward_tiny_workload():
 def test_backward_mid_size_long_window():
     """L=6144, Hq=8, Hkv=2, D=128, W=2048, n_sink=4: several key tiles per band, sinks seen by every later tile."""
     run_forward_backward(inputs.PrefillConfig("bwdmid", (6144,), 8, 2, 128, 2048, 4, False, seed=77))
+
+
+def test_backward_split_sink_tiles_ragged_batch():
+    """Sequences of 4500, 2300 and 70 tokens with 100 sink tokens (two sink key tiles) and W=256: the long sequences
+    take the path where a sink tile's query range is cut over several blocks and dk, dv are summed in fp32; the
+    short one ends inside the first sink tile, and the second chunk of the 2300-token sequence is partly empty."""
+    run_forward_backward(inputs.PrefillConfig("bwdsplit", (4500, 2300, 70), 4, 2, 128, 256, 100, False, seed=91))
