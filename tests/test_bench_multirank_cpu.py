@@ -25,10 +25,17 @@ dist.destroy_process_group()
 """
 
 
+def _free_port():
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
 def _launch(args, env_extra=None, timeout=300):
     env = dict(os.environ, SWAA_ROOT=ROOT, MASTER_ADDR="127.0.0.1", **(env_extra or {}))
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
-           "127.0.0.1", "--master-port", "29531"] + args
+           "127.0.0.1", "--master-port", str(_free_port())] + args
     return subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=timeout, cwd=ROOT)
 
 
