@@ -12,6 +12,7 @@
 #include "swaa_decode.cuh"
 #include "swaa_prefill.cuh"
 #include "swaa_backward.cuh"
+#include "swaa_backward_tc.cuh"
 
 namespace swaa {
 
@@ -431,8 +432,9 @@ struct BackwardWorkspace {
 
 static BackwardWorkspace backward_workspace(int B, int T, int Hq, int Hkv, int D, int n_sink) {
     BackwardWorkspace w;
-    const long long t_rows = ((long long)T + kBwdTile - 1) / kBwdTile * kBwdTile;
-    const long long s_rows = ((long long)n_sink + kBwdTile - 1) / kBwdTile * kBwdTile;
+    // rows of the key tiles that hold sink keys, in whole tiles of the wider of the two kernels
+    const long long t_rows = ((long long)T + kBwdTcKeys - 1) / kBwdTcKeys * kBwdTcKeys;
+    const long long s_rows = ((long long)n_sink + kBwdTcKeys - 1) / kBwdTcKeys * kBwdTcKeys;
     w.sink_rows = (int)(s_rows < t_rows ? s_rows : t_rows);
     w.off_dkv = ((size_t)T * Hq * D * sizeof(float) + 255) / 256 * 256;
     w.zero_bytes = w.off_dkv + 2 * (size_t)B * w.sink_rows * Hkv * D * sizeof(float);
@@ -442,33 +444,44 @@ static BackwardWorkspace backward_workspace(int B, int T, int Hq, int Hkv, int D
     return w;
 }
 
+// D = 128 runs on the tcgen05 kernel (128-key tiles), D = 64 on the warp-level kernel (64-key tiles).
 template <int D>
 static int launch_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
                            const BackwardParams& p, void* dq, int max_seqlen, size_t zero_bytes, cudaStream_t st) {
-    using L = BackwardSmem<D>;
+    constexpr bool kTc = D == 128;
+    constexpr int kKeyTile = kTc ? kBwdTcKeys : kBwdTile;
+    constexpr int kRowTile = kTc ? kBwdTcRows : kBwdTile;
     CUtensorMap tq, tk, tv, tdo;
     int rc;
-    if ((rc = make_token_major_map(&tq, q, p.T, p.Hq, D, kBwdTile)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&tk, k, p.T, p.Hkv, D, kBwdTile)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&tv, v, p.T, p.Hkv, D, kBwdTile)) != SWAA_OK) return rc;
-    if ((rc = make_token_major_map(&tdo, dout, p.T, p.Hq, D, kBwdTile)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tq, q, p.T, p.Hq, D, kRowTile)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tk, k, p.T, p.Hkv, D, kKeyTile)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tv, v, p.T, p.Hkv, D, kKeyTile)) != SWAA_OK) return rc;
+    if ((rc = make_token_major_map(&tdo, dout, p.T, p.Hq, D, kRowTile)) != SWAA_OK) return rc;
     const size_t n_acc = (size_t)p.T * p.Hq * D;
     if (cudaMemsetAsync(p.dq_accum, 0, zero_bytes, st) != cudaSuccess) return SWAA_ERR_CUDA;
     const int rows = p.T * p.Hq;
     backward_delta_kernel<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(dout), p.lse,
         const_cast<float*>(p.delta), const_cast<float*>(p.lse2), p.T, p.Hq);
-    if (cudaFuncSetAttribute(backward_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
-        cudaSuccess)
-        return SWAA_ERR_CUDA;
-    const int ntiles = (max_seqlen + kBwdTile - 1) / kBwdTile;
+    const int ntiles = (max_seqlen + kKeyTile - 1) / kKeyTile;
     const dim3 grid((unsigned)(p.sink_tiles * p.chunks + (ntiles - p.sink_tiles)), (unsigned)p.Hkv, (unsigned)p.B);
-    backward_kernel<D><<<grid, kBwdThreads, L::kDynamicBytes, st>>>(tq, tk, tv, tdo, p);
+    if constexpr (kTc) {
+        if (cudaFuncSetAttribute(backward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 BackwardTcSmem::kDynamicBytes) != cudaSuccess)
+            return SWAA_ERR_CUDA;
+        backward_tc_kernel<<<grid, kBwdTcThreads, BackwardTcSmem::kDynamicBytes, st>>>(tq, tk, tv, tdo, p);
+    } else {
+        using L = BackwardSmem<D>;
+        if (cudaFuncSetAttribute(backward_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
+            cudaSuccess)
+            return SWAA_ERR_CUDA;
+        backward_kernel<D><<<grid, kBwdThreads, L::kDynamicBytes, st>>>(tq, tk, tv, tdo, p);
+    }
     backward_convert_dq_kernel<<<(unsigned)((n_acc / 4 + 255) / 256 + 1), 256, 0, st>>>(
         p.dq_accum, static_cast<__nv_bfloat16*>(dq), n_acc);
     int launches = 3;
     if (p.sink_tiles > 0) {
-        const int sink_rows = p.sink_tiles * kBwdTile;
+        const int sink_rows = p.sink_tiles * kKeyTile;
         const size_t plane = (size_t)p.B * sink_rows * p.Hkv * D;
         backward_convert_dkv_kernel<<<(unsigned)((plane / 4 + 255) / 256), 256, 0, st>>>(
             p.dkv_accum, p.dk, p.dv, p.cu_seqlens, p.B, p.T, sink_rows, p.Hkv, D);
@@ -526,17 +539,18 @@ extern "C" int swaa_prefill_backward(const void* q, const void* k, const void* v
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
     // Key tiles that hold sink keys meet every later query tile: with long sequences their query range is cut
     // into chunks handled by separate blocks, which add dk, dv into the fp32 accumulators.
-    const int ntiles = (max_seqlen + kBwdTile - 1) / kBwdTile;
-    p.chunks = (ntiles + kBwdChunkTiles - 1) / kBwdChunkTiles;
+    const int key_tile = D == 128 ? kBwdTcKeys : kBwdTile;  // the two kernels' key tiles; both step over 64 query rows
+    const int ntiles = (max_seqlen + key_tile - 1) / key_tile;
+    p.chunks = ((max_seqlen + 63) / 64 + kBwdChunkTiles - 1) / kBwdChunkTiles;
     p.sink_tiles = 0;
     if (!is_full && p.chunks > 1) {
-        const int st_need = (int)(((long long)n_sink + kBwdTile - 1) / kBwdTile);
+        const int st_need = (int)(((long long)n_sink + key_tile - 1) / key_tile);
         p.sink_tiles = st_need < ntiles ? st_need : ntiles;
-        if (p.sink_tiles * kBwdTile > w.sink_rows) p.sink_tiles = w.sink_rows / kBwdTile;
+        if (p.sink_tiles * key_tile > w.sink_rows) p.sink_tiles = w.sink_rows / key_tile;
     }
     if (p.sink_tiles == 0) p.chunks = 1;
     if ((long long)p.sink_tiles * p.chunks + (ntiles - p.sink_tiles) > 0x7fffffffLL) return SWAA_ERR_UNSUPPORTED;
-    const size_t zero_bytes = p.sink_tiles > 0 ? w.off_dkv + 2 * (size_t)B * p.sink_tiles * kBwdTile * Hkv * D * sizeof(float)
+    const size_t zero_bytes = p.sink_tiles > 0 ? w.off_dkv + 2 * (size_t)B * p.sink_tiles * key_tile * Hkv * D * sizeof(float)
                                                : (size_t)T * Hq * D * sizeof(float);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     return D == 128 ? launch_backward<128>(q, k, v, out, dout, p, dq, max_seqlen, zero_bytes, st)
