@@ -12,8 +12,9 @@
 //
 // with P^T = exp2(S^T * scale * log2e - lse2[row]) and dS^T = scale * P^T * (dP^T - delta[row]) computed by
 // the thread that owns the key (one tensor-memory lane per key).  dV and dK stay in tensor memory for the
-// whole block; dQ^T is added to an fp32 accumulator in global memory (one coalesced 128-byte reduction per
-// warp and row).  Two groups of four warps take alternate steps, each with its own S^T/dP^T columns, so the
+// whole block; dQ^T goes through shared memory (transposed to [rows][D]) and is added to an fp32 accumulator in
+// global memory by bulk reduce-add copies (per-lane atomics saturate the L2 atomic units and stall the block's
+// other shared-memory traffic behind them).  Two groups of four warps take alternate steps, each with its own S^T/dP^T columns, so the
 // element-wise work of one step overlaps the products of the other.
 //
 // Tensor memory (512 columns): dV [0,128) | dK [128,256) | X_0 [256,384) | X_1 [384,512); X_g holds
@@ -57,10 +58,23 @@ struct BackwardTcSmem {
 // kind::f16 instruction descriptor with both operands read MN-major from shared memory.
 __host__ __device__ constexpr uint32_t make_idesc_mn_mn(int M, int N) { return make_idesc(M, N, 1) | (1u << 15); }
 
+// Vote of the 128 threads of one element-wise group (named barrier `id`): true when `pred` holds for all of them.
+// A bounded wait can give up in one thread and succeed in its neighbour; the vote makes the group leave together,
+// which the plain group barriers further down rely on.
+__device__ __forceinline__ bool group_all(bool pred, int id) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbar.red.and.pred q, %2, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id)
+        : "memory");
+    return r != 0;
+}
+
 __global__ void __launch_bounds__(kBwdTcThreads, 1)
 backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                   const BackwardParams p) {
+                   const __grid_constant__ CUtensorMap tm_dq, const BackwardParams p) {
     using L = BackwardTcSmem;
     constexpr int D = 128, BK = kBwdTcKeys, BR = kBwdTcRows, NQ = kBwdTcStages;
     constexpr uint32_t kIdS = make_idesc(BK, BR, 0);      // S^T, dP^T
@@ -265,8 +279,9 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t ph = (uint32_t)(s >> 1) & 1u;
             const int h = hk * p.G + s / nm, i0 = (m_lo + s % nm) * BR;
             const int i1 = min(i0 + BR, Lseq) - 1;
-            ok = mbar_wait(bar(BAR_QF + st), (uint32_t)(s / NQ) & 1u, abort_flag) &&
-                 mbar_wait(bar(BAR_SF + grp), ph, abort_flag);
+            ok = group_all(mbar_wait(bar(BAR_QF + st), (uint32_t)(s / NQ) & 1u, abort_flag) &&
+                               mbar_wait(bar(BAR_SF + grp), ph, abort_flag),
+                           1 + grp);
             if (!ok) break;
             tc_fence_after();
             const float* rows = s_rows + st * 128;
@@ -314,25 +329,37 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             mbar_arrive(bar(BAR_PR + grp));
 
             // ---- dQ^T of this step: lane = channel, column = row; one 128-byte reduction per warp and row
-            ok = mbar_wait(bar(BAR_DQ + grp), ph, abort_flag);
+            ok = group_all(mbar_wait(bar(BAR_DQ + grp), ph, abort_flag), 1 + grp);
             if (!ok) break;
             tc_fence_after();
-            float* dq_col = p.dq_accum + ((size_t)(seq_start + i0) * p.Hq + h) * D + kl;
+            // 32 rows at a time: registers -> [32 rows][128 channels] fp32 in the group's dS^T buffer (free once dQ^T
+            // is complete) -> one bulk reduce-add of the box into the fp32 accumulator.  Rows of the box past the end
+            // of the sequence receive exact zeros (their dS^T columns are zero); rows past T are clipped by the copy.
             const int nrows = i1 - i0 + 1;
+            const uint32_t stg = sDS + (uint32_t)grp * L::kDSBytes;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                uint32_t v[32];
-                tmem_ld32(tX + 32u * (uint32_t)half, v);
-                tc_wait_ld();
+                if (32 * half < nrows) {
+                    uint32_t v[32];
+                    tmem_ld32(tX + 32u * (uint32_t)half, v);
+                    tc_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const int r = 32 * half + e;
-                    if (r < nrows) atomicAdd(dq_col + (size_t)r * p.Hq * D, __uint_as_float(v[e]));
+                    for (int e = 0; e < 32; ++e)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + (uint32_t)(e * 128 + kl) * 4u), "r"(v[e]) : "memory");
+                    fence_proxy_async_smem();
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+                    if (kl == 0) {
+                        tma_reduce_add_3d(&tm_dq, stg, 0, h, seq_start + i0 + 32 * half);
+                        tma_store_commit();
+                        tma_store_wait_read();  // the staging buffer may be rewritten
+                    }
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
                 }
             }
             tc_fence_before();
             mbar_arrive(bar(BAR_DR + grp));
         }
+        if (kl == 0) tma_store_wait_all();  // this group's reductions into dq have been performed
         // ---- dV (group 0) and dK (group 1) rows of this thread's key
         if (ok) ok = mbar_wait(bar(BAR_FIN), 0u, abort_flag);
         if (ok) {

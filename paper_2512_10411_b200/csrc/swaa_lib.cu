@@ -287,6 +287,20 @@ static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H
     return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
+// fp32 [T][H][D] accumulator, boxes of [rows][1 head][D] without swizzle (target of bulk reduce-add copies).
+static int make_accum_map(CUtensorMap* map, const float* base, int T, int H, int D, int box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return SWAA_ERR_CUDA;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 4, (cuuint64_t)H * D * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)D, 1, (cuuint32_t)box_rows};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
+}
+
 template <int D, int kMode>
 static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                           const PrefillParams& p, int sm_count, cudaStream_t st) {
@@ -469,7 +483,9 @@ static int launch_backward(const void* q, const void* k, const void* v, const vo
         if (cudaFuncSetAttribute(backward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  BackwardTcSmem::kDynamicBytes) != cudaSuccess)
             return SWAA_ERR_CUDA;
-        backward_tc_kernel<<<grid, kBwdTcThreads, BackwardTcSmem::kDynamicBytes, st>>>(tq, tk, tv, tdo, p);
+        CUtensorMap tacc;
+        if ((rc = make_accum_map(&tacc, p.dq_accum, p.T, p.Hq, D, 32)) != SWAA_OK) return rc;
+        backward_tc_kernel<<<grid, kBwdTcThreads, BackwardTcSmem::kDynamicBytes, st>>>(tq, tk, tv, tdo, tacc, p);
     } else {
         using L = BackwardSmem<D>;
         if (cudaFuncSetAttribute(backward_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
