@@ -12,8 +12,8 @@
 //
 // with P^T = exp2(S^T * scale * log2e - lse2[row]) and dS^T = scale * P^T * (dP^T - delta[row]) computed by
 // the thread that owns the key (one tensor-memory lane per key).  dV and dK stay in tensor memory for the
-// whole block; dQ^T goes through shared memory (transposed to [rows][D]) and is added to an fp32 accumulator in
-// global memory by bulk reduce-add copies (per-lane atomics saturate the L2 atomic units and stall the block's
+// whole block; dQ^T goes through shared memory (transposed to [rows][D], in the ring stage of the step's Q and dO
+// tiles, which are dead by then) and is added to an fp32 accumulator in global memory by one bulk reduce-add copy (per-lane atomics saturate the L2 atomic units and stall the block's
 // other shared-memory traffic behind them).  Two groups of four warps take alternate steps, each with its own S^T/dP^T columns, so the
 // element-wise work of one step overlaps the products of the other.
 //
@@ -25,6 +25,8 @@
 // Warps 0-7: the two element-wise groups; warp 8: TMA producer (K, V once; Q, dO and the row terms per
 // step through a ring of three stages); warp 9: MMA issuer.  Every wait is bounded.
 #pragma once
+
+#include <type_traits>
 
 #include "swaa_backward.cuh"
 #include "swaa_prefill.cuh"  // tcgen05 wrappers, descriptors
@@ -243,21 +245,21 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
             for (int s = 0; s < n_steps && ok; ++s) {
                 const int g = s & 1;
-                const uint32_t ph = (uint32_t)(s >> 1) & 1u;
-                ok = mbar_wait(bar(BAR_PR + g), ph, abort_flag);
+                ok = mbar_wait(bar(BAR_PR + g), (uint32_t)(s >> 1) & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 issue_g(s);
                 tc_commit(bar(BAR_DQ + g));
-                tc_commit(bar(BAR_QE + s % NQ));
-                if (s + 2 < n_steps) {
-                    // X_g is free once the group has taken dQ^T of step s out of it
-                    ok = mbar_wait(bar(BAR_DR + g), ph, abort_flag) &&
-                         mbar_wait(bar(BAR_QF + (s + 2) % NQ), (uint32_t)((s + 2) / NQ) & 1u, abort_flag);
+                if (s >= 1 && s + 1 < n_steps) {
+                    // S^T, dP^T of step s + 1 go to the other group's columns, free once that group has taken
+                    // dQ^T of step s - 1 out of them.  (Waiting here for this group's own dQ^T instead would put
+                    // its read-out on the issuer's critical path.)
+                    ok = mbar_wait(bar(BAR_DR + (g ^ 1)), (uint32_t)((s - 1) >> 1) & 1u, abort_flag) &&
+                         mbar_wait(bar(BAR_QF + (s + 1) % NQ), (uint32_t)((s + 1) / NQ) & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_s(s + 2);
-                    tc_commit(bar(BAR_SF + g));
+                    issue_s(s + 1);
+                    tc_commit(bar(BAR_SF + (g ^ 1)));
                 }
             }
             // all products issued by this thread must have retired before the tensor memory is read or freed
@@ -273,7 +275,51 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t lane_bits = (uint32_t)(32 * quad) << 16;
         const uint32_t tX = tmem_base + lane_bits + 256u + 128u * (uint32_t)grp;
         const uint32_t sDSg = sDS + (uint32_t)grp * L::kDSBytes + (uint32_t)kl * 128u;
+        // rows of the step that this key sees: i in [max(j, .), hi) with hi = end of the window (or of the sequence)
+        const int vis_hi = (full || j < p.n_sink) ? Lseq : (int)min((long long)Lseq, (long long)j + p.window);
         bool ok = true;
+        int pending_stage = -1;  // thread kl == 0: ring stage that holds the previous step's dQ staging
+        // One half (32 rows) of the element-wise step; kMask: the tile has pairs outside the mask.
+        auto half_step = [&](auto mask_tag, int half, const float* rows, int i0) {
+            constexpr bool kMask = decltype(mask_tag)::value;
+            uint32_t sv[32], dv[32], pk[16], dk[16];
+            tmem_ld32(tX + 32u * (uint32_t)half, sv);
+            tmem_ld32(tX + 64u + 32u * (uint32_t)half, dv);
+            tc_wait_ld();
+            // visible rows of this half, as offsets: r in [r_lo, r_hi)
+            const int r_lo = j - i0 - 32 * half, r_hi = vis_hi - i0 - 32 * half;
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+                const int r = 32 * half + e;
+                const float4 l4 = *reinterpret_cast<const float4*>(rows + r);
+                const float4 d4 = *reinterpret_cast<const float4*>(rows + 64 + r);
+                const float ls[4] = {l4.x, l4.y, l4.z, l4.w}, ds[4] = {d4.x, d4.y, d4.z, d4.w};
+                float pv[4], dsv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    pv[u] = ex2f(fmaf(__uint_as_float(sv[e + u]), sl2, -ls[u]));
+                    dsv[u] = pv[u] * (__uint_as_float(dv[e + u]) - ds[u]) * p.scale;
+                    if (kMask) {
+                        const bool vis = e + u >= r_lo && e + u < r_hi;
+                        pv[u] = vis ? pv[u] : 0.f;
+                        dsv[u] = vis ? dsv[u] : 0.f;
+                    }
+                }
+                pk[e >> 1] = pack_bf16x2(pv[0], pv[1]);
+                pk[(e >> 1) + 1] = pack_bf16x2(pv[2], pv[3]);
+                dk[e >> 1] = pack_bf16x2(dsv[0], dsv[1]);
+                dk[(e >> 1) + 1] = pack_bf16x2(dsv[2], dsv[3]);
+            }
+            // P^T and dS^T as bf16 pairs over columns that this thread has already read
+            tmem_st16(tX + 16u * (uint32_t)half, pk);
+            tmem_st16(tX + 64u + 16u * (uint32_t)half, dk);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {  // dS^T row of this key: 16-byte chunk 4*half + q, 128-byte swizzle
+                const int ch = 4 * half + q;
+                st_shared_v4(sDSg + (uint32_t)((ch ^ (kl & 7)) << 4), dk[4 * q], dk[4 * q + 1], dk[4 * q + 2],
+                             dk[4 * q + 3]);
+            }
+        };
         for (int s = grp; s < n_steps && ok; s += 2) {
             const int st = s % NQ;
             const uint32_t ph = (uint32_t)(s >> 1) & 1u;
@@ -284,80 +330,53 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                            1 + grp);
             if (!ok) break;
             tc_fence_after();
+            if (kl == 0 && pending_stage >= 0) {
+                // the reduce-add of this group's previous step has read its staging (issued two steps ago): hand
+                // the ring stage back to the producer
+                tma_store_wait_read();
+                mbar_arrive(bar(BAR_QE + pending_stage));
+                pending_stage = -1;
+            }
             const float* rows = s_rows + st * 128;
             const bool need_mask = i0 + BR > Lseq || tile_needs_mask(i0, i1, j0, j1, p.window, p.n_sink, full);
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t sv[32], dv[32], pk[16], dk[16];
-                tmem_ld32(tX + 32u * (uint32_t)half, sv);
-                tmem_ld32(tX + 64u + 32u * (uint32_t)half, dv);
-                tc_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    const int r = 32 * half + e;
-                    const float2 l2 = *reinterpret_cast<const float2*>(rows + r);
-                    const float2 dl = *reinterpret_cast<const float2*>(rows + 64 + r);
-                    float p0 = ex2f(fmaf(__uint_as_float(sv[e]), sl2, -l2.x));
-                    float p1 = ex2f(fmaf(__uint_as_float(sv[e + 1]), sl2, -l2.y));
-                    float d0 = p0 * (__uint_as_float(dv[e]) - dl.x) * p.scale;
-                    float d1 = p1 * (__uint_as_float(dv[e + 1]) - dl.y) * p.scale;
-                    if (need_mask) {
-                        const int ia = i0 + r, ib = ia + 1;
-                        const bool va = ia < Lseq && j <= ia && (full || j > ia - p.window || j < p.n_sink);
-                        const bool vb = ib < Lseq && j <= ib && (full || j > ib - p.window || j < p.n_sink);
-                        p0 = va ? p0 : 0.f;
-                        d0 = va ? d0 : 0.f;
-                        p1 = vb ? p1 : 0.f;
-                        d1 = vb ? d1 : 0.f;
-                    }
-                    pk[e >> 1] = pack_bf16x2(p0, p1);
-                    dk[e >> 1] = pack_bf16x2(d0, d1);
-                }
-                // P^T and dS^T as bf16 pairs over columns that this thread has already read
-                tmem_st16(tX + 16u * (uint32_t)half, pk);
-                tmem_st16(tX + 64u + 16u * (uint32_t)half, dk);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {  // dS^T row of this key: 16-byte chunk 4*half + q, 128-byte swizzle
-                    const int ch = 4 * half + q;
-                    st_shared_v4(sDSg + (uint32_t)((ch ^ (kl & 7)) << 4), dk[4 * q], dk[4 * q + 1], dk[4 * q + 2],
-                                 dk[4 * q + 3]);
-                }
+            if (need_mask) {
+                half_step(std::true_type{}, 0, rows, i0);
+                half_step(std::true_type{}, 1, rows, i0);
+            } else {
+                half_step(std::false_type{}, 0, rows, i0);
+                half_step(std::false_type{}, 1, rows, i0);
             }
             tc_wait_st();
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(bar(BAR_PR + grp));
 
-            // ---- dQ^T of this step: lane = channel, column = row; one 128-byte reduction per warp and row
+            // ---- dQ^T of this step (lane = channel, column = row) -> [64 rows][128 channels] fp32 in the step's
+            // ring stage (Q and dO are no longer needed once dQ^T is complete) -> one bulk reduce-add of the box
+            // into the fp32 accumulator.  Rows of the box past the end of the sequence receive exact zeros (their
+            // dS^T columns are zero); rows past T are clipped by the copy.
             ok = group_all(mbar_wait(bar(BAR_DQ + grp), ph, abort_flag), 1 + grp);
             if (!ok) break;
             tc_fence_after();
-            // 32 rows at a time: registers -> [32 rows][128 channels] fp32 in the group's dS^T buffer (free once dQ^T
-            // is complete) -> one bulk reduce-add of the box into the fp32 accumulator.  Rows of the box past the end
-            // of the sequence receive exact zeros (their dS^T columns are zero); rows past T are clipped by the copy.
-            const int nrows = i1 - i0 + 1;
-            const uint32_t stg = sDS + (uint32_t)grp * L::kDSBytes;
+            const uint32_t stg = sRing + (uint32_t)st * L::kStageBytes + (uint32_t)kl * 4u;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                if (32 * half < nrows) {
-                    uint32_t v[32];
-                    tmem_ld32(tX + 32u * (uint32_t)half, v);
-                    tc_wait_ld();
+                uint32_t v[32];
+                tmem_ld32(tX + 32u * (uint32_t)half, v);
+                tc_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + (uint32_t)(e * 128 + kl) * 4u), "r"(v[e]) : "memory");
-                    fence_proxy_async_smem();
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
-                    if (kl == 0) {
-                        tma_reduce_add_3d(&tm_dq, stg, 0, h, seq_start + i0 + 32 * half);
-                        tma_store_commit();
-                        tma_store_wait_read();  // the staging buffer may be rewritten
-                    }
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
-                }
+                for (int e = 0; e < 32; ++e)
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + (uint32_t)((32 * half + e) * 512)), "r"(v[e]) : "memory");
             }
             tc_fence_before();
-            mbar_arrive(bar(BAR_DR + grp));
+            mbar_arrive(bar(BAR_DR + grp));  // the group's columns may take the next S^T, dP^T
+            fence_proxy_async_smem();
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+            if (kl == 0) {
+                tma_reduce_add_3d(&tm_dq, sRing + (uint32_t)st * L::kStageBytes, 0, h, seq_start + i0);
+                tma_store_commit();
+                pending_stage = st;
+            }
         }
         if (kl == 0) tma_store_wait_all();  // this group's reductions into dq have been performed
         // ---- dV (group 0) and dK (group 1) rows of this thread's key

@@ -484,7 +484,7 @@ static int launch_backward(const void* q, const void* k, const void* v, const vo
                                  BackwardTcSmem::kDynamicBytes) != cudaSuccess)
             return SWAA_ERR_CUDA;
         CUtensorMap tacc;
-        if ((rc = make_accum_map(&tacc, p.dq_accum, p.T, p.Hq, D, 32)) != SWAA_OK) return rc;
+        if ((rc = make_accum_map(&tacc, p.dq_accum, p.T, p.Hq, D, kBwdTcRows)) != SWAA_OK) return rc;
         backward_tc_kernel<<<grid, kBwdTcThreads, BackwardTcSmem::kDynamicBytes, st>>>(tq, tk, tv, tdo, tacc, p);
     } else {
         using L = BackwardSmem<D>;
