@@ -23,7 +23,7 @@
 // makes these overlays safe.
 //
 // Warps 0-7: the two element-wise groups; warp 8: TMA producer (K, V once; Q, dO and the row terms per
-// step through a ring of three stages); warp 9: MMA issuer.  Every wait is bounded.
+// step through a ring of four stages); warp 9: MMA issuer.  Every wait is bounded.
 #pragma once
 
 #include <type_traits>
@@ -36,7 +36,7 @@ namespace swaa {
 constexpr int kBwdTcKeys = 128;    // keys per block
 constexpr int kBwdTcRows = 64;     // query rows per step
 constexpr int kBwdTcThreads = 320;
-constexpr int kBwdTcStages = 3;    // ring of (Q, dO, row terms)
+constexpr int kBwdTcStages = 4;    // ring of (Q, dO, row terms); a stage also stages the step's dQ on its way out
 
 struct BackwardTcSmem {
     static constexpr int D = 128;
@@ -54,7 +54,8 @@ struct BackwardTcSmem {
     static constexpr int kNumBars = 1 + 2 * kBwdTcStages + 4 * 2 + 1;
     static constexpr int kOffMisc = kOffBar + kNumBars * 8;
     static constexpr int kBytes = kOffMisc + 32;
-    static constexpr int kDynamicBytes = kBytes + 1024;
+    static constexpr int kDynamicBytes = kBytes;  // the kernel declares the array 1024-byte aligned and checks it
+    static_assert(kDynamicBytes <= 232448, "shared memory per block");
 };
 
 // kind::f16 instruction descriptor with both operands read MN-major from shared memory.
@@ -83,9 +84,13 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     constexpr uint32_t kIdKV = make_idesc(BK, D, 1);      // dV, dK (A from tensor memory)
     constexpr uint32_t kIdDQ = make_idesc_mn_mn(D, BR);   // dQ^T
 
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t smem_base = smem_u32(smem_raw);
+    uint8_t* smem_gen = smem_raw;
+    if ((smem_base & 1023u) != 0u) {  // the swizzled tiles need it; uniform, before any barrier or allocation
+        if (threadIdx.x == 0) record_device_error(SWAA_ERR_CUDA);
+        return;
+    }
     const uint32_t sK = smem_base + L::kOffK, sV = smem_base + L::kOffV, sRing = smem_base + L::kOffRing;
     const uint32_t sDS = smem_base + L::kOffDS;
     float* s_rows = reinterpret_cast<float*>(smem_gen + L::kOffRows);
@@ -208,14 +213,22 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t ds_t0 = (uint32_t)smem_desc_sw128(sDS, 16, 1024);                 // dS^T of group 0, MN-major (B)
             constexpr uint32_t kStageStep = (uint32_t)L::kStageBytes >> 4, kDoStep = (uint32_t)L::kQTileBytes >> 4;
             constexpr uint32_t kDsStep = (uint32_t)L::kDSBytes >> 4;
-            // S^T and dP^T of step s into X_{s & 1}
-            auto issue_s = [&](int s) {
+            // S^T = K Q^T (columns [0,64) of X_{s & 1}) and dP^T = V dO^T (columns [64,128)) of step s
+            auto issue_st = [&](int s) {
                 const uint32_t qb = q_b0 + (uint32_t)(s % NQ) * kStageStep, tX = tmem_base + 256u + 128u * (uint32_t)(s & 1);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t oa = ((uint32_t)(kk >> 2) * L::kKVPanelBytes + (uint32_t)(kk & 3) * 32u) >> 4;
                     const uint32_t ob = ((uint32_t)(kk >> 2) * L::kQPanelBytes + (uint32_t)(kk & 3) * 32u) >> 4;
                     mma_ss_lh(tX, k_a + oa, qb + ob, hi, kIdS, kk > 0 ? 1u : 0u);
+                }
+            };
+            auto issue_dp = [&](int s) {
+                const uint32_t qb = q_b0 + (uint32_t)(s % NQ) * kStageStep, tX = tmem_base + 256u + 128u * (uint32_t)(s & 1);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t oa = ((uint32_t)(kk >> 2) * L::kKVPanelBytes + (uint32_t)(kk & 3) * 32u) >> 4;
+                    const uint32_t ob = ((uint32_t)(kk >> 2) * L::kQPanelBytes + (uint32_t)(kk & 3) * 32u) >> 4;
                     mma_ss_lh(tX + 64u, v_a + oa, qb + kDoStep + ob, hi, kIdS, kk > 0 ? 1u : 0u);
                 }
             };
@@ -240,26 +253,30 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ok = mbar_wait(bar(BAR_QF + s % NQ), 0u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                issue_s(s);
+                issue_dp(s);
+                issue_st(s);
                 tc_commit(bar(BAR_SF + s));
             }
+            // Steady state: G(s) as soon as the group has written P^T, dS^T of step s; then the products that feed
+            // the same group's step s + 2.  dP^T(s+2) only needs columns [64,128), free once G(s) has run (products
+            // run in issue order); S^T(s+2) overwrites dQ^T(s) and waits until the group has taken it out.
             for (int s = 0; s < n_steps && ok; ++s) {
                 const int g = s & 1;
-                ok = mbar_wait(bar(BAR_PR + g), (uint32_t)(s >> 1) & 1u, abort_flag);
+                const uint32_t ph = (uint32_t)(s >> 1) & 1u;
+                ok = mbar_wait(bar(BAR_PR + g), ph, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 issue_g(s);
                 tc_commit(bar(BAR_DQ + g));
-                if (s >= 1 && s + 1 < n_steps) {
-                    // S^T, dP^T of step s + 1 go to the other group's columns, free once that group has taken
-                    // dQ^T of step s - 1 out of them.  (Waiting here for this group's own dQ^T instead would put
-                    // its read-out on the issuer's critical path.)
-                    ok = mbar_wait(bar(BAR_DR + (g ^ 1)), (uint32_t)((s - 1) >> 1) & 1u, abort_flag) &&
-                         mbar_wait(bar(BAR_QF + (s + 1) % NQ), (uint32_t)((s + 1) / NQ) & 1u, abort_flag);
+                if (s + 2 < n_steps) {
+                    ok = mbar_wait(bar(BAR_QF + (s + 2) % NQ), (uint32_t)((s + 2) / NQ) & 1u, abort_flag);
+                    if (!ok) break;
+                    issue_dp(s + 2);
+                    ok = mbar_wait(bar(BAR_DR + g), ph, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_s(s + 1);
-                    tc_commit(bar(BAR_SF + (g ^ 1)));
+                    issue_st(s + 2);
+                    tc_commit(bar(BAR_SF + g));
                 }
             }
             // all products issued by this thread must have retired before the tensor memory is read or freed
