@@ -401,6 +401,20 @@ def run_profile_case(case: str):
         out = torch.empty_like(q)
         for _ in range(3):
             swaa.swaa_prefill(q, k, v, out, cu, cfg.seqlens[0], cfg.window, cfg.n_sink, cfg.is_full)
+    elif case == "backward":
+        # heads and mask of workload 2 at a quarter of its length (0.5 GB on the device with the fp32 workspace)
+        cfg = inputs.PrefillConfig("backward_L8192", (8192,), 32, 8, 128, 2048, 4, False, seed=2)
+        q, k, v, cu = inputs.make_prefill_inputs(cfg, "cuda")
+        T, Hq, D = q.shape
+        out, dout = torch.empty_like(q), torch.randn(q.shape, device="cuda").to(torch.bfloat16)
+        lse = torch.empty((Hq, T), dtype=torch.float32, device="cuda")
+        swaa.swaa_prefill(q, k, v, out, cu, cfg.seqlens[0], cfg.window, cfg.n_sink, False, lse=lse)
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        ws = torch.empty(swaa.prefill_backward_workspace_size(1, T, Hq, cfg.Hkv, D, cfg.n_sink), dtype=torch.uint8,
+                         device="cuda")
+        for _ in range(3):
+            swaa.swaa_prefill_backward(q, k, v, out, dout, lse, cu, cfg.seqlens[0], cfg.window, cfg.n_sink, False, dq, dk,
+                                       dv, ws)
     else:
         cfg = inputs.cfg_decode(B=4) if case.endswith("_small") else inputs.cfg_decode()
         full = "fa" in case
@@ -616,8 +630,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--profile-case", default=None,
-                    choices=["prefill", "prefill_full", "prefill_tiny", "decode_fa", "decode_swa", "decode_fa_small",
-                             "decode_swa_small"],
+                    choices=["prefill", "prefill_full", "prefill_tiny", "backward", "decode_fa", "decode_swa",
+                             "decode_fa_small", "decode_swa_small"],
                     help="run three launches of one kernel only (for ncu) and exit")
     ap.add_argument("--sweep", action="store_true",
                     help="time swaa_prefill on the other workloads and the L / W / n_sink sweeps (one GPU) and exit")
