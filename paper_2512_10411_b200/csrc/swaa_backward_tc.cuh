@@ -259,7 +259,10 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
             // Steady state: G(s) as soon as the group has written P^T, dS^T of step s; then the products that feed
             // the same group's step s + 2.  dP^T(s+2) only needs columns [64,128), free once G(s) has run (products
-            // run in issue order); S^T(s+2) overwrites dQ^T(s) and waits until the group has taken it out.
+            // run in issue order), and fills the time until the group has taken dQ^T(s) out of the columns that
+            // S^T(s+2) overwrites.  (Every look at a barrier costs this thread about 80 cycles during which no
+            // product is issued; folding the tile barrier into the group's arrival was slower all the same, because
+            // dP^T then waits for the read-out too.)
             for (int s = 0; s < n_steps && ok; ++s) {
                 const int g = s & 1;
                 const uint32_t ph = (uint32_t)(s >> 1) & 1u;
@@ -269,6 +272,8 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 issue_g(s);
                 tc_commit(bar(BAR_DQ + g));
                 if (s + 2 < n_steps) {
+                    // one wait for both: the group arrives after it has taken dQ^T(s) out of its columns and has
+                    // seen the tiles of step s + 2 land
                     ok = mbar_wait(bar(BAR_QF + (s + 2) % NQ), (uint32_t)((s + 2) / NQ) & 1u, abort_flag);
                     if (!ok) break;
                     issue_dp(s + 2);
@@ -376,17 +381,20 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             const uint32_t stg = sRing + (uint32_t)st * L::kStageBytes + (uint32_t)kl * 4u;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t v[32];
-                tmem_ld32(tX + 32u * (uint32_t)half, v);
+            {
+                uint32_t v0[32], v1[32];
+                tmem_ld32(tX, v0);
+                tmem_ld32(tX + 32u, v1);
                 tc_wait_ld();
+                // the group's columns may take the next S^T as soon as dQ^T is in registers
+                tc_fence_before();
+                mbar_arrive(bar(BAR_DR + grp));
 #pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + (uint32_t)((32 * half + e) * 512)), "r"(v[e]) : "memory");
+                for (int e = 0; e < 32; ++e) {
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + (uint32_t)(e * 512)), "r"(v0[e]) : "memory");
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + (uint32_t)((32 + e) * 512)), "r"(v1[e]) : "memory");
+                }
             }
-            tc_fence_before();
-            mbar_arrive(bar(BAR_DR + grp));  // the group's columns may take the next S^T, dP^T
             fence_proxy_async_smem();
             asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
             if (kl == 0) {
