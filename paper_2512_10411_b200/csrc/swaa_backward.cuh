@@ -60,11 +60,12 @@ struct BackwardSmem {
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
 
-// delta[h, t] = sum_d out[t, h, d] * dout[t, h, d]; one warp per (t, h).
+// delta[h, t] = sum_d out[t, h, d] * dout[t, h, d] and lse2 = lse * log2(e); one warp per (t, h), which also clears
+// its row of the fp32 dq accumulator.
 template <int D>
 __global__ void backward_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
                                       const float* __restrict__ lse, float* __restrict__ delta,
-                                      float* __restrict__ lse2, int T, int Hq) {
+                                      float* __restrict__ lse2, float* __restrict__ dq_accum, int T, int Hq) {
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (row >= T * Hq) return;
     const int t = row / Hq, h = row - t * Hq;
@@ -76,6 +77,8 @@ __global__ void backward_delta_kernel(const __nv_bfloat16* __restrict__ out, con
         const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(g + d));
         acc += a.x * b.x + a.y * b.y;
     }
+    for (int d = lane * 4; d < D; d += 128)
+        *reinterpret_cast<float4*>(dq_accum + (size_t)row * D + d) = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (lane == 0) {
         delta[(size_t)h * T + t] = acc;

@@ -461,7 +461,7 @@ static BackwardWorkspace backward_workspace(int B, int T, int Hq, int Hkv, int D
 // D = 128 runs on the tcgen05 kernel (128-key tiles), D = 64 on the warp-level kernel (64-key tiles).
 template <int D>
 static int launch_backward(const void* q, const void* k, const void* v, const void* out, const void* dout,
-                           const BackwardParams& p, void* dq, int max_seqlen, size_t zero_bytes, cudaStream_t st) {
+                           const BackwardParams& p, void* dq, int max_seqlen, size_t dkv_zero_bytes, cudaStream_t st) {
     constexpr bool kTc = D == 128;
     constexpr int kKeyTile = kTc ? kBwdTcKeys : kBwdTile;
     constexpr int kRowTile = kTc ? kBwdTcRows : kBwdTile;
@@ -472,11 +472,12 @@ static int launch_backward(const void* q, const void* k, const void* v, const vo
     if ((rc = make_token_major_map(&tv, v, p.T, p.Hkv, D, kKeyTile)) != SWAA_OK) return rc;
     if ((rc = make_token_major_map(&tdo, dout, p.T, p.Hq, D, kRowTile)) != SWAA_OK) return rc;
     const size_t n_acc = (size_t)p.T * p.Hq * D;
-    if (cudaMemsetAsync(p.dq_accum, 0, zero_bytes, st) != cudaSuccess) return SWAA_ERR_CUDA;
+    // the dq accumulator is cleared by the kernel that computes the row terms; the (small) dk, dv accumulators here
+    if (dkv_zero_bytes > 0 && cudaMemsetAsync(p.dkv_accum, 0, dkv_zero_bytes, st) != cudaSuccess) return SWAA_ERR_CUDA;
     const int rows = p.T * p.Hq;
     backward_delta_kernel<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(dout), p.lse,
-        const_cast<float*>(p.delta), const_cast<float*>(p.lse2), p.T, p.Hq);
+        const_cast<float*>(p.delta), const_cast<float*>(p.lse2), p.dq_accum, p.T, p.Hq);
     const int ntiles = (max_seqlen + kKeyTile - 1) / kKeyTile;
     const dim3 grid((unsigned)(p.sink_tiles * p.chunks + (ntiles - p.sink_tiles)), (unsigned)p.Hkv, (unsigned)p.B);
     if constexpr (kTc) {
@@ -566,11 +567,10 @@ extern "C" int swaa_prefill_backward(const void* q, const void* k, const void* v
     }
     if (p.sink_tiles == 0) p.chunks = 1;
     if ((long long)p.sink_tiles * p.chunks + (ntiles - p.sink_tiles) > 0x7fffffffLL) return SWAA_ERR_UNSUPPORTED;
-    const size_t zero_bytes = p.sink_tiles > 0 ? w.off_dkv + 2 * (size_t)B * p.sink_tiles * key_tile * Hkv * D * sizeof(float)
-                                               : (size_t)T * Hq * D * sizeof(float);
+    const size_t dkv_zero_bytes = 2 * (size_t)B * p.sink_tiles * key_tile * Hkv * D * sizeof(float);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return D == 128 ? launch_backward<128>(q, k, v, out, dout, p, dq, max_seqlen, zero_bytes, st)
-                    : launch_backward<64>(q, k, v, out, dout, p, dq, max_seqlen, zero_bytes, st);
+    return D == 128 ? launch_backward<128>(q, k, v, out, dout, p, dq, max_seqlen, dkv_zero_bytes, st)
+                    : launch_backward<64>(q, k, v, out, dout, p, dq, max_seqlen, dkv_zero_bytes, st);
 }
 
 // ------------------------------------------------------------------------------------ lazy ratio
