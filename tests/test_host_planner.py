@@ -144,3 +144,16 @@ def test_trimmed_cache_holds_exactly_the_visible_keys():
             want = {j for j in range(n) if oracle.visible(n - 1, j, W, S, False)}
             assert set(slots.values()) == want, (W, S, n)
     assert swaa.trimmed_cache_slot(-1, 4, 0) == -1 and swaa.trimmed_cache_len(5, 0, 0) == -1
+
+
+def test_backward_workspace_size_covers_its_parts(_lib):
+    """The backward workspace holds an fp32 dq accumulator, two fp32 row terms per (head, token) and fp32 dk/dv rows
+    for the key tiles that hold sink keys (whole tiles of 128 rows, at most the packed length)."""
+    size = swaa.prefill_backward_workspace_size
+    B, T, Hq, Hkv, D = 3, 5000, 8, 2, 128
+    base = T * Hq * D * 4 + 2 * Hq * T * 4
+    assert base <= size(B, T, Hq, Hkv, D, 0) <= base + 3 * 256
+    for n_sink, rows in ((1, 128), (128, 128), (129, 256), (10 ** 6, 5120)):
+        want = base + 2 * B * rows * Hkv * D * 4
+        assert want <= size(B, T, Hq, Hkv, D, n_sink) <= want + 3 * 256, n_sink
+    assert size(0, T, Hq, Hkv, D, 4) == 256 and size(B, T, Hq, Hkv, D, -1) == 256  # invalid shapes: the minimum
