@@ -90,6 +90,8 @@ SMALL = [
     ((257, 640), 3, 1, 128),   # three query heads per kv head
     ((200, 333), 2, 2, 64),
     ((63,), 8, 2, 128),
+    ((40, 64, 65, 200), 2, 2, 128),  # one query head per kv head: blocks with a single step
+    ((130, 1), 8, 1, 128),           # eight query heads per kv head
 ]
 POLICIES = [(1, 0, True), (1, 0, False), (64, 0, False), (128, 4, False), (100, 7, False), (65, 70, False),
             (300, 1, False), (4096, 4, False)]
