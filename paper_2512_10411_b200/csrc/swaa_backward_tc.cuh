@@ -10,7 +10,7 @@
 //   dK  += dS^T Q    [128 keys x D]         A = dS^T in tensor memory,        B = Q tile read MN-major
 //   dQ^T = K^T dS^T  [D x 64 rows]          A = K tile read MN-major, B = dS^T in shared memory (MN-major)
 //
-// with P^T = exp2(S^T * scale * log2e - lse2[row]) and dS^T = scale * P^T * (dP^T - delta[row]) computed by
+// with P^T = exp2(S^T * scale * log2e - lse2[row]) and dS^T = P^T * (scale * dP^T - scale * delta[row]) computed by
 // the thread that owns the key (one tensor-memory lane per key).  dV and dK stay in tensor memory for the
 // whole block; dQ^T goes through shared memory (transposed to [rows][D], in the ring stage of the step's Q and dO
 // tiles, which are dead by then) and is added to an fp32 accumulator in global memory by one bulk reduce-add copy (per-lane atomics saturate the L2 atomic units and stall the block's
@@ -183,10 +183,11 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
             }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {  // 64 x lse2, 64 x delta; zeros past the end of the sequence
+            for (int q = 0; q < 4; ++q) {  // 64 x lse2, 64 x delta (negated, delta scaled); zeros past the end of the sequence
                 const int idx = lane + 32 * q, r = idx & 63, i = i0 + r;
                 const float* src = (idx < 64 ? p.lse2 : p.delta) + (size_t)h * p.T + seq_start;
-                s_rows[st * 128 + idx] = i < Lseq ? src[i] : 0.f;
+                // stored ready for one fused multiply-add each: -lse2 and -delta * scale
+                s_rows[st * 128 + idx] = i < Lseq ? -src[i] * (idx < 64 ? 1.f : p.scale) : 0.f;
             }
             mbar_arrive(bar(BAR_QF + st));
             issued = s + 1;
@@ -302,6 +303,7 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         bool ok = true;
         int pending_stage = -1;  // thread kl == 0: ring stage that holds the previous step's dQ staging
         // One half (32 rows) of the element-wise step; kMask: the tile has pairs outside the mask.
+        const uint64_t sl2x2 = pack_f32x2(sl2, sl2), scx2 = pack_f32x2(p.scale, p.scale);
         auto half_step = [&](auto mask_tag, int half, const float* rows, int i0) {
             constexpr bool kMask = decltype(mask_tag)::value;
             uint32_t sv[32], dv[32], pk[16], dk[16];
@@ -313,15 +315,26 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
                 const int r = 32 * half + e;
-                const float4 l4 = *reinterpret_cast<const float4*>(rows + r);
-                const float4 d4 = *reinterpret_cast<const float4*>(rows + 64 + r);
-                const float ls[4] = {l4.x, l4.y, l4.z, l4.w}, ds[4] = {d4.x, d4.y, d4.z, d4.w};
+                const float4 l4 = *reinterpret_cast<const float4*>(rows + r);       // -lse2 of four rows
+                const float4 d4 = *reinterpret_cast<const float4*>(rows + 64 + r);  // -delta * scale
                 float pv[4], dsv[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    pv[u] = ex2f(fmaf(__uint_as_float(sv[e + u]), sl2, -ls[u]));
-                    dsv[u] = pv[u] * (__uint_as_float(dv[e + u]) - ds[u]) * p.scale;
-                    if (kMask) {
+                for (int u = 0; u < 4; u += 2) {  // two rows per packed fp32 instruction
+                    const uint64_t x = fma_f32x2(pack_f32x2(__uint_as_float(sv[e + u]), __uint_as_float(sv[e + u + 1])), sl2x2,
+                                                 u ? pack_f32x2(l4.z, l4.w) : pack_f32x2(l4.x, l4.y));
+                    const uint64_t t = fma_f32x2(pack_f32x2(__uint_as_float(dv[e + u]), __uint_as_float(dv[e + u + 1])), scx2,
+                                                 u ? pack_f32x2(d4.z, d4.w) : pack_f32x2(d4.x, d4.y));
+                    float x0, x1;
+                    unpack_f32x2(x, x0, x1);
+                    pv[u] = ex2f(x0);
+                    pv[u + 1] = ex2f(x1);
+                    uint64_t d2;
+                    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d2) : "l"(pack_f32x2(pv[u], pv[u + 1])), "l"(t));
+                    unpack_f32x2(d2, dsv[u], dsv[u + 1]);
+                }
+                if (kMask) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
                         const bool vis = e + u >= r_lo && e + u < r_hi;
                         pv[u] = vis ? pv[u] : 0.f;
                         dsv[u] = vis ? dsv[u] : 0.f;
