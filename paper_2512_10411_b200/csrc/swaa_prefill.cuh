@@ -552,8 +552,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     const bool has_next = n + 1 < nt;
                     const int sk = (g + 1) % ST;
                     const uint32_t pk = (uint32_t)((g + 1) / ST) & 1u;
-                    ok = mbar_wait(bar(BAR_PR + 0), (uint32_t)gs[0] & 1u, abort_flag) &&
-                         mbar_wait(bar(BAR_VF + sv), pv, abort_flag);
+                    // The tiles first (they landed long ago as a rule), then the side's P: a look at a barrier costs
+                    // this thread some 80 cycles even when it has completed, and what follows the P barrier is on
+                    // the side's critical path softmax -> PV -> QK -> softmax.
+                    ok = mbar_wait(bar(BAR_VF + sv), pv, abort_flag) &&
+                         (!has_next || mbar_wait(bar(BAR_KF + sk), pk, abort_flag)) &&
+                         mbar_wait(bar(BAR_PR + 0), (uint32_t)gs[0] & 1u, abort_flag);
                     if (kPaged && ok && w.k_off + w.seq_len - trng.tile(n) * BN < BN) {
                         // last key tile of a sequence that ends inside it: the producer clears the rows past the end
                         ok = mbar_wait(bar(BAR_VC), (uint32_t)n_cleared & 1u, abort_flag);
@@ -567,9 +571,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     tc_commit(bar(BAR_OD + 0));
                     ++gs[0];
                     if (has_next) {
-                        ok = mbar_wait(bar(BAR_KF + sk), pk, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
                         issue_qk(0, sk);
                         tc_commit(bar(BAR_SF + 0));
                     }
