@@ -568,7 +568,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(0, sv, n > 0);
-                    tc_commit(bar(BAR_OD + 0));
+                    // O-done is only waited for by the item's epilogue: between tiles the S-full barrier of tile n + 1
+                    // already implies PV(n) (a commit covers every product issued before it), and every commit costs
+                    // this thread some 40 cycles
+                    if (!has_next) tc_commit(bar(BAR_OD + 0));
                     ++gs[0];
                     if (has_next) {
                         issue_qk(0, sk);
@@ -581,7 +584,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         if (!ok) break;
                         tc_fence_after();
                         issue_pv(1, sv, n > 0);
-                        tc_commit(bar(BAR_OD + 1));
+                        if (!has_next) tc_commit(bar(BAR_OD + 1));
                         ++gs[1];
                         if (has_next) {
                             issue_qk(1, sk);
@@ -613,7 +616,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
         const uint32_t tS = tmem_base + lane_base + (uint32_t)side * 128u;
         const uint32_t tO = tmem_base + lane_base + 256u + (uint32_t)side * (uint32_t)D;
-        int gs = 0;  // tiles processed by this side so far
+        int gs = 0;          // tiles processed by this side so far
+        int items_done = 0;  // items finished by this side (phase of O-done)
         bool ok = true;
         for (int it = 0; ok; ++it) {
             WorkItem w;
@@ -681,10 +685,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const float m_new = fmaxf(m_used, rmax);
                 const bool need = (m_used != -INFINITY) && ((m_new - m_used) * p.sl2 > kRescaleThreshold);
                 if (__any_sync(0xffffffffu, need)) {
-                    // raise the reference maximum of every row of this warp and rescale O accordingly
-                    ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(gs - 1) & 1u, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
+                    // raise the reference maximum of every row of this warp and rescale O accordingly; PV of the
+                    // previous tile has completed: it was issued before the QK whose S-full barrier this warp passed
                     const float alpha = (m_used == -INFINITY) ? 1.f : ex2f((m_used - m_new) * p.sl2);
 #pragma unroll
                     for (int cc = 0; cc < D / 32; ++cc) {
@@ -759,8 +761,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             if (!ok) break;
             // ---- epilogue of this item: O / l -> bf16 -> global
             SWAA_TICK(e0);
-            ok = mbar_wait(bar(BAR_OD + side), (uint32_t)(gs - 1) & 1u, abort_flag);
+            ok = mbar_wait(bar(BAR_OD + side), (uint32_t)items_done & 1u, abort_flag);
             if (!ok) break;
+            ++items_done;
             tc_fence_after();
             uint32_t orr[D];
 #pragma unroll
