@@ -273,8 +273,7 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 issue_g(s);
                 tc_commit(bar(BAR_DQ + g));
                 if (s + 2 < n_steps) {
-                    // one wait for both: the group arrives after it has taken dQ^T(s) out of its columns and has
-                    // seen the tiles of step s + 2 land
+                    // (this look falls under the tail of G(s); ahead of the wait for the group it was slower)
                     ok = mbar_wait(bar(BAR_QF + (s + 2) % NQ), (uint32_t)((s + 2) / NQ) & 1u, abort_flag);
                     if (!ok) break;
                     issue_dp(s + 2);
