@@ -35,7 +35,7 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists).
-PREFILL_DRAM_TRAFFIC_BYTES = 639519488  # 404.52 MB read + 235.00 MB written, profiles/prefill_kernel_cfg2_long_swa.txt
+PREFILL_DRAM_TRAFFIC_BYTES = 642869504  # 404.54 MB read + 238.33 MB written, profiles/prefill_kernel_cfg2_long_swa.txt
 
 # decode kernel: 4 x (1.0739 GB read + 4 MB written) scaled from the B=4 capture; 270.0 MB + 5 MB at full size
 DECODE_FA_DRAM_TRAFFIC_BYTES = 4 * (1073919000 + 4249600)
