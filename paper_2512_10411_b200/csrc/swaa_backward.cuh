@@ -9,7 +9,11 @@
 //     dQ_i   = scale * sum_j dS_ij k_j,   dK_j = scale * sum_i dS_ij q_i
 // with dK, dV summed over the query heads of a GQA group.
 //
-// One thread block owns one 64-key tile of one (sequence, key/value head) and keeps its dK and dV in
+// This file holds the parts shared by the two kernels (parameters, the row-term and conversion kernels) and
+// the warp-level kernel used for head dimension 64; head dimension 128 runs on the tcgen05 kernel of
+// swaa_backward_tc.cuh.
+//
+// Warp-level kernel: one thread block owns one 64-key tile of one (sequence, key/value head) and keeps its dK and dV in
 // registers; it walks the query heads of the group and, per head, only the 64-row query tiles that can
 // see the key tile (the band above it, plus every later tile when the key tile holds sink keys), so the
 // work is O(L * window) like the forward pass (App. A).  Each of the four warps owns 16 keys: it forms
@@ -17,7 +21,9 @@
 // tensor-core MMAs (fp32 accumulation), feeds P^T and dS^T straight back as A operands for
 // dV += P^T dO and dK += dS^T Q, and leaves dS^T in shared memory, from where every warp takes the 16
 // query rows it owns to form dQ += dS K; dQ is accumulated across key tiles in an fp32 buffer with
-// atomic adds and converted to bf16 by a second kernel.  Tiles are staged by TMA (128-byte swizzle).
+// atomic adds and converted to bf16 by a second kernel.  Tiles are staged by TMA (128-byte swizzle).  The key
+// tiles that hold sink keys meet every later query tile: with long sequences their query range is cut into
+// chunks handled by separate blocks, which add dK and dV into fp32 accumulators (converted by a third kernel).
 #pragma once
 
 #include "swaa_internal.cuh"
