@@ -126,3 +126,28 @@ def test_backward_split_sink_tiles_ragged_batch():
     take the path where a sink tile's query range is cut over several blocks and dk, dv are summed in fp32; the
     short one ends inside the first sink tile, and the second chunk of the 2300-token sequence is partly empty."""
     run_forward_backward(inputs.PrefillConfig("bwdsplit", (4500, 2300, 70), 4, 2, 128, 256, 100, False, seed=91))
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_backward_reports_bad_cu_seqlens_and_argument_errors(D):
+    """Both kernels: a cu_seqlens that runs past T is reported through the status word and the call returns; host-side
+    checks (workspace too small, unsupported head size, window < 1) are refused before any launch."""
+    cfg = inputs.PrefillConfig("bwdbad", (256, 256), 4, 2, D, 16, 2, False, seed=63)
+    q, k, v, cu = inputs.make_prefill_inputs(cfg, "cuda")
+    T, Hq, _ = q.shape
+    out, dout = torch.zeros_like(q), torch.ones_like(q)
+    lse = torch.zeros((Hq, T), dtype=torch.float32, device="cuda")
+    dq, dk, dv = torch.zeros_like(q), torch.zeros_like(k), torch.zeros_like(v)
+    ws = torch.empty(swaa.prefill_backward_workspace_size(2, T, Hq, cfg.Hkv, D, 2), dtype=torch.uint8, device="cuda")
+    assert swaa.last_device_status() == 0
+    bad = torch.tensor([0, 300, 600], dtype=torch.int32, device="cuda")  # second sequence ends past T = 512
+    swaa.swaa_prefill_backward(q, k, v, out, dout, lse, bad, 300, 16, 2, False, dq, dk, dv, ws)
+    assert swaa.last_device_status() == -5
+    swaa.swaa_prefill_backward(q, k, v, out, dout, lse, cu, 256, 16, 2, False, dq, dk, dv, ws)
+    assert swaa.last_device_status() == 0
+    with pytest.raises(swaa.SwaaError) as e:
+        swaa.swaa_prefill_backward(q, k, v, out, dout, lse, cu, 256, 16, 2, False, dq, dk, dv, ws[:1024])
+    assert e.value.status == -4
+    with pytest.raises(swaa.SwaaError) as e:
+        swaa.swaa_prefill_backward(q, k, v, out, dout, lse, cu, 256, 0, 2, False, dq, dk, dv, ws)
+    assert e.value.status == -1
