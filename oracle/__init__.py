@@ -16,6 +16,7 @@ from .swaa_oracle import (  # noqa: F401
     prefill,
     prefill_backward,
     prefill_backward_c,
+    prefill_backward_rows,
     prefill_chunked,
     prefill_paged,
     visible,

@@ -141,7 +141,11 @@ int swaa_oracle_prefill(const float* q, const float* k, const float* v, const in
         for (int64_t r = 0; r < n_rows; ++r) {
             int64_t t = row_t ? row_t[r] : r / Hq;
             int h = row_t ? row_h[r] : (int)(r % Hq);
-            if (t < 0 || t >= T || h < 0 || h >= Hq) { bad = 1; continue; }
+            if (t < 0 || t >= T || h < 0 || h >= Hq) {
+#pragma omp atomic write
+                bad = 1;
+                continue;
+            }
             int b = 0;
             while (!(cu_seqlens[b] <= t && t < cu_seqlens[b + 1])) ++b; /* sequence that owns token t */
             int64_t start = cu_seqlens[b];
@@ -189,7 +193,11 @@ int swaa_oracle_prefill_chunked(const float* q, const float* k, const float* v, 
         for (int64_t r = 0; r < n_rows; ++r) {
             int64_t t = row_t ? row_t[r] : r / Hq;
             int h = row_t ? row_h[r] : (int)(r % Hq);
-            if (t < 0 || t >= Tq || h < 0 || h >= Hq) { bad = 1; continue; }
+            if (t < 0 || t >= Tq || h < 0 || h >= Hq) {
+#pragma omp atomic write
+                bad = 1;
+                continue;
+            }
             int b = 0;
             while (!(cu_q[b] <= t && t < cu_q[b + 1])) ++b; /* sequence that owns query token t */
             int64_t lq = (int64_t)cu_q[b + 1] - cu_q[b], lk = (int64_t)cu_k[b + 1] - cu_k[b];
@@ -239,7 +247,7 @@ int swaa_oracle_decode(const float* q, const float* kcache, const float* vcache,
 
 /*
  * Gradients of the packed self-attention prefill with respect to q, k, v for an upstream gradient dout
- * (Sec. 3.3: fine-tuning under the SWA mask).  From out_i = sum_j p_ij v_j, p = softmax over the visible keys
+ * (Sec. 3.2.2: fine-tuning under the SWA mask).  From out_i = sum_j p_ij v_j, p = softmax over the visible keys
  * of s_ij = scale * q_i.k_j:
  *     dv_j += p_ij dout_i;   dp_ij = dout_i . v_j;   ds_ij = p_ij (dp_ij - sum_j' p_ij' dp_ij');
  *     dq_i = scale * sum_j ds_ij k_j;   dk_j += scale * ds_ij q_i     (dk, dv summed over the heads of a group).
@@ -349,6 +357,147 @@ int swaa_oracle_prefill_backward(const float* q, const float* k, const float* v,
             }
         }
     }
+    free(rm);
+    free(rden);
+    free(rdot);
+    return 0;
+}
+
+/*
+ * The same gradients for chosen rows and keys only, so that a long sequence can be checked without the
+ * O(L * W) cost of every row (Sec. 3.2.2; formulas as in swaa_oracle_prefill_backward, nothing else changes):
+ *   dq for the n_q (packed token, query head) pairs (qrow_t[r], qrow_h[r])      -> dq_out [n_q, D]
+ *   dk, dv for the n_k (packed token, key/value head) pairs (key_t[r], key_hk[r]) -> dk_out, dv_out [n_k, D]
+ * A key's gradient needs the softmax statistics (maximum, denominator, sum_j p_ij dp_ij) of every row that
+ * sees it, for all query heads of its group; those are computed once for exactly the rows that some chosen key
+ * needs, each by the same two plain passes over its visible keys, and then used by the key loop.
+ * Returns 0, or -1 on inconsistent arguments.
+ */
+int swaa_oracle_prefill_backward_rows(const float* q, const float* k, const float* v, const float* dout,
+                                      const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D, int64_t W, int64_t S,
+                                      int is_full, double scale, int64_t n_q, const int64_t* qrow_t,
+                                      const int32_t* qrow_h, double* dq_out, int64_t n_k, const int64_t* key_t,
+                                      const int32_t* key_hk, double* dk_out, double* dv_out) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
+    if (!is_full && W < 1) return -1;
+    if (S < 0 || n_q < 0 || n_k < 0) return -1;
+    const int G = Hq / Hkv;
+    const int64_t T = B > 0 ? cu_seqlens[B] : 0;
+    int64_t max_len = 0;
+    for (int b = 0; b < B; ++b) {
+        int64_t len = (int64_t)cu_seqlens[b + 1] - cu_seqlens[b];
+        if (len < 0) return -1;
+        if (len > max_len) max_len = len;
+    }
+    for (int64_t r = 0; r < n_q; ++r)
+        if (qrow_t[r] < 0 || qrow_t[r] >= T || qrow_h[r] < 0 || qrow_h[r] >= Hq) return -1;
+    for (int64_t r = 0; r < n_k; ++r)
+        if (key_t[r] < 0 || key_t[r] >= T || key_hk[r] < 0 || key_hk[r] >= Hkv) return -1;
+    /* which (token, kv head) rows does some chosen key need the statistics of? */
+    unsigned char* need = (unsigned char*)calloc((size_t)(T * Hkv > 0 ? T * Hkv : 1), 1);
+    for (int64_t r = 0; r < n_k; ++r) {
+        const int64_t t = key_t[r];
+        int b = 0;
+        while (!(cu_seqlens[b] <= t && t < cu_seqlens[b + 1])) ++b;
+        const int64_t s0 = cu_seqlens[b], len = cu_seqlens[b + 1] - s0, j = t - s0;
+        for (int64_t i = j; i < len; ++i)
+            if (swaa_oracle_visible(i, j, W, S, is_full)) need[(s0 + i) * Hkv + key_hk[r]] = 1;
+    }
+    double* rm = (double*)malloc(sizeof(double) * (size_t)(T * Hq > 0 ? T * Hq : 1));
+    double* rden = (double*)malloc(sizeof(double) * (size_t)(T * Hq > 0 ? T * Hq : 1));
+    double* rdot = (double*)malloc(sizeof(double) * (size_t)(T * Hq > 0 ? T * Hq : 1));
+#pragma omp parallel
+    {
+        double* sc = (double*)malloc(sizeof(double) * (size_t)(max_len > 0 ? max_len : 1));
+        double* dp = (double*)malloc(sizeof(double) * (size_t)(max_len > 0 ? max_len : 1));
+        /* pass A: statistics of the needed rows (r < T*Hq), then dq of the chosen rows (r >= T*Hq) */
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t r = 0; r < T * Hq + n_q; ++r) {
+            const int chosen = r >= T * Hq;
+            const int64_t t = chosen ? qrow_t[r - T * Hq] : r / Hq;
+            const int h = chosen ? qrow_h[r - T * Hq] : (int)(r % Hq);
+            const int hk = h / G;
+            if (!chosen && !need[t * Hkv + hk]) continue;
+            int b = 0;
+            while (!(cu_seqlens[b] <= t && t < cu_seqlens[b + 1])) ++b;
+            const int64_t s0 = cu_seqlens[b], i = t - s0;
+            const float* qi = q + (t * Hq + h) * (int64_t)D;
+            const float* gi = dout + (t * Hq + h) * (int64_t)D;
+            double m = -INFINITY;
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                const float* kj = k + ((s0 + j) * Hkv + hk) * (int64_t)D;
+                const float* vj = v + ((s0 + j) * Hkv + hk) * (int64_t)D;
+                double s = 0.0, d = 0.0;
+                for (int c = 0; c < D; ++c) {
+                    s += (double)qi[c] * (double)kj[c];
+                    d += (double)gi[c] * (double)vj[c];
+                }
+                sc[j] = s * scale;
+                dp[j] = d;
+                if (sc[j] > m) m = sc[j];
+            }
+            double den = 0.0, dot = 0.0;
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                den += exp(sc[j] - m);
+            }
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                dot += exp(sc[j] - m) / den * dp[j];
+            }
+            if (!chosen) {
+                rm[r] = m;
+                rden[r] = den;
+                rdot[r] = dot;
+                continue;
+            }
+            double* dqi = dq_out + (r - T * Hq) * D;
+            for (int c = 0; c < D; ++c) dqi[c] = 0.0;
+            for (int64_t j = 0; j <= i; ++j) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                const double ds = exp(sc[j] - m) / den * (dp[j] - dot);
+                const float* kj = k + ((s0 + j) * Hkv + hk) * (int64_t)D;
+                for (int c = 0; c < D; ++c) dqi[c] += scale * ds * (double)kj[c];
+            }
+        }
+        free(sc);
+        free(dp);
+        /* pass B: the chosen keys collect from the rows and heads that see them */
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t r = 0; r < n_k; ++r) {
+            const int64_t t = key_t[r];
+            const int hk = key_hk[r];
+            int b = 0;
+            while (!(cu_seqlens[b] <= t && t < cu_seqlens[b + 1])) ++b;
+            const int64_t s0 = cu_seqlens[b], len = cu_seqlens[b + 1] - s0, j = t - s0;
+            const float* kj = k + (t * Hkv + hk) * (int64_t)D;
+            const float* vj = v + (t * Hkv + hk) * (int64_t)D;
+            double* dkj = dk_out + r * D;
+            double* dvj = dv_out + r * D;
+            for (int c = 0; c < D; ++c) dkj[c] = dvj[c] = 0.0;
+            for (int64_t i = j; i < len; ++i) {
+                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                for (int h = hk * G; h < (hk + 1) * G; ++h) {
+                    const int64_t ri = (s0 + i) * Hq + h;
+                    const float* qi = q + ri * D;
+                    const float* gi = dout + ri * D;
+                    double s = 0.0, d = 0.0;
+                    for (int c = 0; c < D; ++c) {
+                        s += (double)qi[c] * (double)kj[c];
+                        d += (double)gi[c] * (double)vj[c];
+                    }
+                    const double p = exp(s * scale - rm[ri]) / rden[ri];
+                    const double ds = p * (d - rdot[ri]);
+                    for (int c = 0; c < D; ++c) {
+                        dvj[c] += p * (double)gi[c];
+                        dkj[c] += scale * ds * (double)qi[c];
+                    }
+                }
+            }
+        }
+    }
+    free(need);
     free(rm);
     free(rden);
     free(rdot);

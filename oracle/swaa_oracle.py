@@ -51,6 +51,9 @@ def _load():
         lib.swaa_oracle_prefill_backward.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
                                                      vp, vp, vp]
         lib.swaa_oracle_prefill_backward.restype = ctypes.c_int
+        lib.swaa_oracle_prefill_backward_rows.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int,
+                                                          dbl, i64, vp, vp, vp, i64, vp, vp, vp, vp]
+        lib.swaa_oracle_prefill_backward_rows.restype = ctypes.c_int
         lib.swaa_oracle_decode.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
                                            vp, vp, vp, vp]
         lib.swaa_oracle_decode.restype = ctypes.c_int
@@ -264,6 +267,34 @@ def prefill_backward_c(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_f
                                               _ptr(dk), _ptr(dv))
     if rc != 0:
         raise ValueError("swaa_oracle_prefill_backward: inconsistent arguments")
+    return {"dq": dq, "dk": dk, "dv": dv}
+
+
+def prefill_backward_rows(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_full: bool, q_rows, kv_rows,
+                          scale: float | None = None):
+    """Gradients for chosen rows and keys only (plain-C loops, same formulas as prefill_backward_c): dq for the
+    (packed token, query head) pairs q_rows = (t, h) and dk, dv for the (packed token, kv head) pairs kv_rows =
+    (t, hk).  Returns dq [n_q, D], dk, dv [n_k, D] float64."""
+    q, k, v, dout = _f32(q), _f32(k), _f32(v), _f32(dout)
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    qt = np.ascontiguousarray(np.asarray(q_rows[0], dtype=np.int64))
+    qh = np.ascontiguousarray(np.asarray(q_rows[1], dtype=np.int32))
+    kt = np.ascontiguousarray(np.asarray(kv_rows[0], dtype=np.int64))
+    kh = np.ascontiguousarray(np.asarray(kv_rows[1], dtype=np.int32))
+    assert qt.shape == qh.shape and kt.shape == kh.shape
+    dq = np.empty((qt.shape[0], D), dtype=np.float64)
+    dk = np.empty((kt.shape[0], D), dtype=np.float64)
+    dv = np.empty((kt.shape[0], D), dtype=np.float64)
+    rc = _load().swaa_oracle_prefill_backward_rows(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(cu), cu.shape[0] - 1, Hq,
+                                                   Hkv, D, int(window), int(n_sink), int(bool(is_full)), float(scale),
+                                                   qt.shape[0], _ptr(qt), _ptr(qh), _ptr(dq), kt.shape[0], _ptr(kt),
+                                                   _ptr(kh), _ptr(dk), _ptr(dv))
+    if rc != 0:
+        raise ValueError("swaa_oracle_prefill_backward_rows: inconsistent arguments")
     return {"dq": dq, "dk": dk, "dv": dv}
 
 

@@ -133,6 +133,43 @@ def test_paged_decode_honours_the_block_table():
         assert np.array_equal(a["out"], d["out"]) and np.isfinite(a["out"]).all()
 
 
+def test_paged_prefill_honours_the_block_table():
+    """The twin of the paged-decode pin for prefill_paged: packed contexts scattered over pages handed out in random
+    order, unused pages and the rows past each sequence's last key poisoned with NaN.  The result must be the
+    chunked prefill of the packed copy, bit for bit; a swapped j // page_size and j % page_size, a block-table row
+    taken from the wrong sequence or a read past seqlens_k would surface as a mismatch or a NaN."""
+    rng = np.random.default_rng(12)
+    Hq, Hkv, D, page = 4, 2, 16, 8
+    lq, lk = [5, 29, 1, 8], [29, 29, 17, 8]
+    B, max_blocks, num_pages = len(lk), 5, 40
+    ks = [_bf16_randn((n, Hkv, D), 80 + b) for b, n in enumerate(lk)]
+    vs = [_bf16_randn((n, Hkv, D), 90 + b) for b, n in enumerate(lk)]
+    q = _bf16_randn((sum(lq), Hq, D), 79)
+    kp = np.full((num_pages, page, Hkv, D), np.nan, dtype=np.float32)
+    vp = np.full_like(kp, np.nan)
+    perm = rng.permutation(num_pages)
+    bt = np.full((B, max_blocks), -1, dtype=np.int32)
+    nxt = 0
+    for b in range(B):
+        for blk in range((lk[b] + page - 1) // page):
+            pg = perm[nxt]; nxt += 1
+            bt[b, blk] = pg
+            n = min(page, lk[b] - blk * page)
+            kp[pg, :n] = ks[b][blk * page:blk * page + n]
+            vp[pg, :n] = vs[b][blk * page:blk * page + n]
+    cq, ck = np.concatenate([[0], np.cumsum(lq)]), np.concatenate([[0], np.cumsum(lk)])
+    for W, S, full in ((6, 2, False), (3, 0, False), (1, 0, True)):
+        a = oracle.prefill_paged(q, kp, vp, cq, lk, bt, W, S, full)
+        d = oracle.prefill_chunked(q, np.concatenate(ks), np.concatenate(vs), cq, ck, W, S, full)
+        for key in ("out", "lse", "nvis"):
+            assert np.array_equal(a[key], d[key]), key
+        assert np.isfinite(a["out"]).all()
+    rows = (np.array([0, 7, 33, 42]), np.array([3, 0, 1, 2], dtype=np.int32))
+    a = oracle.prefill_paged(q, kp, vp, cq, lk, bt, 6, 2, False, rows=rows)
+    d = oracle.prefill_chunked(q, np.concatenate(ks), np.concatenate(vs), cq, ck, 6, 2, False)
+    assert np.array_equal(a["out"], d["out"][rows[0], rows[1]])
+
+
 def test_lazy_ratio_closed_forms():
     """Q = 0 makes the softmax uniform: the share of the recent and sink keys is a count ratio.  A recent window
     that covers the whole context gives 1.  Scores that single out one old key give (almost) 0."""
@@ -189,3 +226,41 @@ def test_backward_matches_autograd_of_a_dense_masked_attention(W, S, full):
     for name, t in (("dq", tq), ("dk", tk), ("dv", tv)):
         assert np.allclose(got[name], t.grad.numpy(), rtol=0, atol=1e-11), name
         assert np.allclose(fast[name], t.grad.numpy(), rtol=0, atol=1e-11), name + " (C loops)"
+
+
+@pytest.mark.parametrize("W,S,full", [(5, 0, False), (4, 2, False), (1, 0, True)])
+def test_backward_rows_equals_autograd_on_the_chosen_rows_and_keys(W, S, full):
+    """The row- and key-sampled gradients (used to check long sequences) against torch.autograd through a dense
+    masked attention, for rows and keys that include sinks, the first and last token of each sequence and
+    repeats; and against the all-rows functions."""
+    lens, Hq, Hkv, D, scale = [11, 1, 17], 4, 2, 8, 0.41
+    T = sum(lens)
+    q, k, v = _bf16_randn((T, Hq, D), 170), _bf16_randn((T, Hkv, D), 171), _bf16_randn((T, Hkv, D), 172)
+    dout = _bf16_randn((T, Hq, D), 173)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    tq, tk, tv = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (q, k, v))
+    outs = []
+    for b, n in enumerate(lens):
+        s0 = int(cu[b])
+        i, j = torch.arange(n)[:, None], torch.arange(n)[None, :]
+        mask = (j <= i) & (torch.tensor(full) | (j > i - W) | (j < S))
+        kk = tk[s0:s0 + n].repeat_interleave(Hq // Hkv, dim=1)
+        vv = tv[s0:s0 + n].repeat_interleave(Hq // Hkv, dim=1)
+        sc = torch.einsum("ihd,jhd->hij", tq[s0:s0 + n], kk) * scale
+        sc = sc.masked_fill(~mask[None], float("-inf"))
+        outs.append(torch.einsum("hij,jhd->ihd", torch.softmax(sc, dim=-1), vv))
+    torch.cat(outs).backward(torch.tensor(dout, dtype=torch.float64))
+    q_rows = (np.array([0, 10, 11, 12, 28, 5, 5]), np.array([0, 3, 1, 2, 3, 1, 1]))
+    kv_rows = (np.array([0, 1, 10, 11, 12, 13, 28, 20, 20]), np.array([0, 1, 1, 0, 1, 0, 1, 0, 0]))
+    got = oracle.prefill_backward_rows(q, k, v, dout, cu, W, S, full, q_rows, kv_rows, scale=scale)
+    assert np.allclose(got["dq"], tq.grad.numpy()[q_rows], rtol=0, atol=1e-11)
+    assert np.allclose(got["dk"], tk.grad.numpy()[kv_rows], rtol=0, atol=1e-11)
+    assert np.allclose(got["dv"], tv.grad.numpy()[kv_rows], rtol=0, atol=1e-11)
+    every = oracle.prefill_backward_c(q, k, v, dout, cu, W, S, full, scale=scale)
+    assert np.allclose(got["dq"], every["dq"][q_rows], rtol=0, atol=1e-13)
+    assert np.allclose(got["dk"], every["dk"][kv_rows], rtol=0, atol=1e-13)
+    assert np.allclose(got["dv"], every["dv"][kv_rows], rtol=0, atol=1e-13)
+    empty = (np.zeros(0, dtype=np.int64), np.zeros(0, dtype=np.int32))
+    assert oracle.prefill_backward_rows(q, k, v, dout, cu, W, S, full, empty, empty)["dq"].shape == (0, D)
+    with pytest.raises(ValueError):
+        oracle.prefill_backward_rows(q, k, v, dout, cu, W, S, full, (np.array([T]), np.array([0])), empty)
