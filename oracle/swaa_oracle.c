@@ -253,11 +253,15 @@ int swaa_oracle_decode(const float* q, const float* kcache, const float* vcache,
  *     dq_i = scale * sum_j ds_ij k_j;   dk_j += scale * ds_ij q_i     (dk, dv summed over the heads of a group).
  * Two plain passes: rows (softmax statistics and dq), then keys (dk, dv from the rows that see them).
  *   q, dout [T, Hq, D]; k, v [T, Hkv, D] float32 (bf16 values); dq [T, Hq, D], dk, dv [T, Hkv, D] double.
+ * out_given (nullable, [T, Hq, D] float32): since out_i = sum_j p_ij v_j, the row term sum_j' p_ij' dp_ij' equals
+ * dout_i . out_i.  With out_given == NULL it is computed from the probabilities (the exact gradient).  With a
+ * tensor given, dout_i . out_given_i is used instead: the gradient as a function of a stored (e.g. rounded) forward
+ * output, which is what an entry point that receives `out` as an argument computes.
  * Returns 0, or -1 on inconsistent arguments.
  */
 int swaa_oracle_prefill_backward(const float* q, const float* k, const float* v, const float* dout,
-                                 const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D, int64_t W, int64_t S,
-                                 int is_full, double scale, double* dq, double* dk, double* dv) {
+                                 const float* out_given, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D,
+                                 int64_t W, int64_t S, int is_full, double scale, double* dq, double* dk, double* dv) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
     if (!is_full && W < 1) return -1;
     if (S < 0) return -1;
@@ -305,9 +309,14 @@ int swaa_oracle_prefill_backward(const float* q, const float* k, const float* v,
                 if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
                 den += exp(sc[j] - m);
             }
-            for (int64_t j = 0; j <= i; ++j) {
-                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
-                dot += exp(sc[j] - m) / den * dp[j];
+            if (out_given) {
+                const float* oi = out_given + (t * Hq + h) * (int64_t)D;
+                for (int c = 0; c < D; ++c) dot += (double)gi[c] * (double)oi[c];
+            } else {
+                for (int64_t j = 0; j <= i; ++j) {
+                    if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                    dot += exp(sc[j] - m) / den * dp[j];
+                }
             }
             rm[r] = m;
             rden[r] = den;
@@ -371,10 +380,11 @@ int swaa_oracle_prefill_backward(const float* q, const float* k, const float* v,
  * A key's gradient needs the softmax statistics (maximum, denominator, sum_j p_ij dp_ij) of every row that
  * sees it, for all query heads of its group; those are computed once for exactly the rows that some chosen key
  * needs, each by the same two plain passes over its visible keys, and then used by the key loop.
+ * out_given as in swaa_oracle_prefill_backward.
  * Returns 0, or -1 on inconsistent arguments.
  */
 int swaa_oracle_prefill_backward_rows(const float* q, const float* k, const float* v, const float* dout,
-                                      const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D, int64_t W, int64_t S,
+                                      const float* out_given, const int32_t* cu_seqlens, int B, int Hq, int Hkv, int D, int64_t W, int64_t S,
                                       int is_full, double scale, int64_t n_q, const int64_t* qrow_t,
                                       const int32_t* qrow_h, double* dq_out, int64_t n_k, const int64_t* key_t,
                                       const int32_t* key_hk, double* dk_out, double* dv_out) {
@@ -442,9 +452,14 @@ int swaa_oracle_prefill_backward_rows(const float* q, const float* k, const floa
                 if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
                 den += exp(sc[j] - m);
             }
-            for (int64_t j = 0; j <= i; ++j) {
-                if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
-                dot += exp(sc[j] - m) / den * dp[j];
+            if (out_given) {
+                const float* oi = out_given + (t * Hq + h) * (int64_t)D;
+                for (int c = 0; c < D; ++c) dot += (double)gi[c] * (double)oi[c];
+            } else {
+                for (int64_t j = 0; j <= i; ++j) {
+                    if (!swaa_oracle_visible(i, j, W, S, is_full)) continue;
+                    dot += exp(sc[j] - m) / den * dp[j];
+                }
             }
             if (!chosen) {
                 rm[r] = m;

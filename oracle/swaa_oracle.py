@@ -48,11 +48,11 @@ def _load():
         lib.swaa_oracle_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
                                                     i64, vp, vp, vp, vp, vp, vp]
         lib.swaa_oracle_prefill_chunked.restype = ctypes.c_int
-        lib.swaa_oracle_prefill_backward.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
-                                                     vp, vp, vp]
+        lib.swaa_oracle_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int,
+                                                     dbl, vp, vp, vp]
         lib.swaa_oracle_prefill_backward.restype = ctypes.c_int
-        lib.swaa_oracle_prefill_backward_rows.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int,
-                                                          dbl, i64, vp, vp, vp, i64, vp, vp, vp, vp]
+        lib.swaa_oracle_prefill_backward_rows.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64,
+                                                          ctypes.c_int, dbl, i64, vp, vp, vp, i64, vp, vp, vp, vp]
         lib.swaa_oracle_prefill_backward_rows.restype = ctypes.c_int
         lib.swaa_oracle_decode.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
                                            vp, vp, vp, vp]
@@ -250,10 +250,16 @@ def prefill_paged(q, kpages, vpages, cu_seqlens_q, seqlens_k, block_table, windo
                            rows)
 
 
-def prefill_backward_c(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_full: bool, scale: float | None = None):
+def prefill_backward_c(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_full: bool, scale: float | None = None,
+                       out_given=None):
     """The same gradients as prefill_backward from the plain-C loops of swaa_oracle.c (fast enough for the sizes of
-    the GPU parity tests).  Returns dq [T,Hq,D], dk, dv [T,Hkv,D] float64."""
+    the GPU parity tests).  Returns dq [T,Hq,D], dk, dv [T,Hkv,D] float64.
+
+    out_given (optional, [T,Hq,D]): take the row term sum_j p_ij dp_ij as dout_i . out_given_i, i.e. the gradient as
+    a function of a stored forward output (see swaa_oracle.c); None: the exact gradient."""
     q, k, v, dout = _f32(q), _f32(k), _f32(v), _f32(dout)
+    og = None if out_given is None else _f32(out_given)
+    assert og is None or og.shape == q.shape
     T, Hq, D = q.shape
     Hkv = k.shape[1]
     cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
@@ -262,7 +268,7 @@ def prefill_backward_c(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_f
     dq = np.empty((T, Hq, D), dtype=np.float64)
     dk = np.empty((T, Hkv, D), dtype=np.float64)
     dv = np.empty((T, Hkv, D), dtype=np.float64)
-    rc = _load().swaa_oracle_prefill_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(cu), cu.shape[0] - 1, Hq, Hkv, D,
+    rc = _load().swaa_oracle_prefill_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(og), _ptr(cu), cu.shape[0] - 1, Hq, Hkv, D,
                                               int(window), int(n_sink), int(bool(is_full)), float(scale), _ptr(dq),
                                               _ptr(dk), _ptr(dv))
     if rc != 0:
@@ -271,11 +277,13 @@ def prefill_backward_c(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_f
 
 
 def prefill_backward_rows(q, k, v, dout, cu_seqlens, window: int, n_sink: int, is_full: bool, q_rows, kv_rows,
-                          scale: float | None = None):
+                          scale: float | None = None, out_given=None):
     """Gradients for chosen rows and keys only (plain-C loops, same formulas as prefill_backward_c): dq for the
     (packed token, query head) pairs q_rows = (t, h) and dk, dv for the (packed token, kv head) pairs kv_rows =
-    (t, hk).  Returns dq [n_q, D], dk, dv [n_k, D] float64."""
+    (t, hk).  out_given as in prefill_backward_c.  Returns dq [n_q, D], dk, dv [n_k, D] float64."""
     q, k, v, dout = _f32(q), _f32(k), _f32(v), _f32(dout)
+    og = None if out_given is None else _f32(out_given)
+    assert og is None or og.shape == q.shape
     T, Hq, D = q.shape
     Hkv = k.shape[1]
     cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
@@ -289,7 +297,7 @@ def prefill_backward_rows(q, k, v, dout, cu_seqlens, window: int, n_sink: int, i
     dq = np.empty((qt.shape[0], D), dtype=np.float64)
     dk = np.empty((kt.shape[0], D), dtype=np.float64)
     dv = np.empty((kt.shape[0], D), dtype=np.float64)
-    rc = _load().swaa_oracle_prefill_backward_rows(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(cu), cu.shape[0] - 1, Hq,
+    rc = _load().swaa_oracle_prefill_backward_rows(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(og), _ptr(cu), cu.shape[0] - 1, Hq,
                                                    Hkv, D, int(window), int(n_sink), int(bool(is_full)), float(scale),
                                                    qt.shape[0], _ptr(qt), _ptr(qh), _ptr(dq), kt.shape[0], _ptr(kt),
                                                    _ptr(kh), _ptr(dk), _ptr(dv))

@@ -264,3 +264,45 @@ def test_backward_rows_equals_autograd_on_the_chosen_rows_and_keys(W, S, full):
     assert oracle.prefill_backward_rows(q, k, v, dout, cu, W, S, full, empty, empty)["dq"].shape == (0, D)
     with pytest.raises(ValueError):
         oracle.prefill_backward_rows(q, k, v, dout, cu, W, S, full, (np.array([T]), np.array([0])), empty)
+
+
+def test_backward_with_a_given_forward_output():
+    """The row term may be taken from a stored forward output (dout . out) instead of the probabilities.  With the
+    exact output both routes are the same gradient; with a perturbed output the difference is, to first order, the
+    closed form  d(dq_i) = -scale * (dout_i . e_i) * sum_j p_ij k_j,  d(dk_j) = -scale * sum_i p_ij (dout_i . e_i) q_i
+    and dv does not move: this pins which tensor enters the dot product, and with which sign."""
+    lens, Hq, Hkv, D, W, S, scale = [13, 6], 4, 2, 8, 5, 2, 0.33
+    T = sum(lens)
+    q, k, v = _bf16_randn((T, Hq, D), 180), _bf16_randn((T, Hkv, D), 181), _bf16_randn((T, Hkv, D), 182)
+    dout = _bf16_randn((T, Hq, D), 183)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    fwd = oracle.prefill(q, k, v, cu, W, S, False, scale=scale)["out"]
+    exact = oracle.prefill_backward_c(q, k, v, dout, cu, W, S, False, scale=scale)
+    same = oracle.prefill_backward_c(q, k, v, dout, cu, W, S, False, scale=scale, out_given=fwd)
+    for n in ("dq", "dk", "dv"):
+        assert np.allclose(same[n], exact[n], rtol=0, atol=2e-6), n  # float32 copy of the exact output
+    e = np.float32(1e-2) * _bf16_randn((T, Hq, D), 184)
+    og = fwd.astype(np.float32) + e
+    moved = oracle.prefill_backward_c(q, k, v, dout, cu, W, S, False, scale=scale, out_given=og)
+    assert np.array_equal(moved["dv"], same["dv"])
+    de = ((og.astype(np.float64) - fwd.astype(np.float32).astype(np.float64)) * dout).sum(-1)  # [T, Hq]
+    G = Hq // Hkv
+    want_dq, want_dk = np.zeros((T, Hq, D)), np.zeros((T, Hkv, D))
+    for b, n in enumerate(lens):
+        s0 = int(cu[b])
+        for i in range(n):
+            keys = np.array(_visible_positions(i, W, S, False)) + s0
+            for h in range(Hq):
+                sc = (k[keys, h // G].astype(np.float64) @ q[s0 + i, h].astype(np.float64)) * scale
+                p = np.exp(sc - sc.max())
+                p /= p.sum()
+                want_dq[s0 + i, h] = -scale * de[s0 + i, h] * (p @ k[keys, h // G].astype(np.float64))
+                want_dk[keys, h // G] += -scale * de[s0 + i, h] * np.outer(p, q[s0 + i, h].astype(np.float64))
+    assert np.allclose(moved["dq"] - same["dq"], want_dq, rtol=0, atol=1e-12)
+    assert np.allclose(moved["dk"] - same["dk"], want_dk, rtol=0, atol=1e-12)
+    rows = (np.array([0, 5, 12, 13, 18]), np.array([0, 1, 2, 3, 0]))
+    keys_ = (np.array([0, 1, 7, 13, 18]), np.array([0, 1, 1, 0, 1]))
+    part = oracle.prefill_backward_rows(q, k, v, dout, cu, W, S, False, rows, keys_, scale=scale, out_given=og)
+    assert np.allclose(part["dq"], moved["dq"][rows], rtol=0, atol=1e-13)
+    assert np.allclose(part["dk"], moved["dk"][keys_], rtol=0, atol=1e-13)
+    assert np.allclose(part["dv"], moved["dv"][keys_], rtol=0, atol=1e-13)
