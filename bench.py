@@ -178,6 +178,45 @@ def max_over_ranks(values, world, device=None):
     return t.tolist()
 
 
+def stats_ms(values):
+    """median / min / mean of a list of per-launch times (ms)."""
+    v = sorted(values)
+    n = len(v)
+    med = v[n // 2] if n % 2 else 0.5 * (v[n // 2 - 1] + v[n // 2])
+    return {"median": med, "min": v[0], "mean": sum(v) / n, "n": n}
+
+
+def time_prefill_case(swaa, torch, flush_l2, stream, peaks, cfg, is_full, reps, tensors=None, sustained=False):
+    """One swaa_prefill workload: `reps` timed launches after one warm-up, L2 flushed before each, CUDA events
+    on the launching stream.  Returns a dict with median / min time and effective throughput."""
+    from paper_2512_10411_b200 import inputs
+
+    q, k, v, cu = tensors if tensors is not None else inputs.make_prefill_inputs(cfg, "cuda")
+    out = torch.empty_like(q)
+    ms = []
+    for r in range(reps + 1):
+        flush_l2()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        swaa.swaa_prefill(q, k, v, out, cu, max(cfg.seqlens), cfg.window, cfg.n_sink, is_full)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if r > 0:
+            ms.append(a.elapsed_time(b))
+    if swaa.last_device_status() != 0:
+        raise RuntimeError("swaa_prefill reported a device error")
+    st = stats_ms(ms)
+    pairs = sum(visible_pairs(L, cfg.window, cfg.n_sink, is_full) for L in cfg.seqlens)
+    flops = 4.0 * cfg.D * cfg.Hq * pairs
+    tf = flops / (st["median"] * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    del out
+    return {"seqlens": list(cfg.seqlens) if len(cfg.seqlens) > 1 else cfg.seqlens[0], "Hq": cfg.Hq, "Hkv": cfg.Hkv,
+            "D": cfg.D, "window": cfg.window, "n_sink": cfg.n_sink, "is_full": bool(is_full), "ms": st["median"],
+            "ms_min": st["min"], "launches": st["n"], "effective_tflops": tf, "frac_of_measured_peak": tf / peak,
+            "frac_of_nominal_2250": tf / 2250.0, "us_per_1k_tokens": 1e3 * st["median"] / (sum(cfg.seqlens) / 1024.0)}
+
+
 def whole_job_value(units_per_rank, n_ranks, seconds):
     """Throughput of the whole job: the units all ranks processed over the slowest rank's time."""
     return n_ranks * units_per_rank / seconds
@@ -278,9 +317,13 @@ def run_ours(args, rank, local_rank, world):
     launches = swaa.kernel_launch_count() - launches0
     assert swaa.last_device_status() == 0
     total_ms = t_start.elapsed_time(t_end)
-    t_pre = sum(e[0].elapsed_time(e[1]) for e in events)
-    t_fa = sum(e[2].elapsed_time(e[3]) for e in events)
-    t_swa = sum(e[4].elapsed_time(e[5]) for e in events)
+    pre_ms = [e[0].elapsed_time(e[1]) for e in events]
+    fa_ms = [e[2].elapsed_time(e[3]) for e in events]
+    swa_ms = [e[4].elapsed_time(e[5]) for e in events]
+    # per kernel: the median over the timed steps is the reported time (a single slow launch, e.g. one that met a
+    # clock change, does not move it); minimum and mean go into the line beside it
+    st_pre, st_fa, st_swa = stats_ms(pre_ms), stats_ms(fa_ms), stats_ms(swa_ms)
+    t_pre, t_fa, t_swa = st_pre["median"], st_fa["median"], st_swa["median"]
 
     # ---------------------------------------------------------------- end to end from host buffers
     qh, kh, vh = (t.cpu().pin_memory() for t in (q, k, v))
@@ -320,6 +363,11 @@ def run_ours(args, rank, local_rank, world):
     total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms = max_over_ranks(
         [total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms], world, dev)
     K, N = args.steps, world
+
+    # ---------------------------------------------------------------- the other workloads and the L sweep (N = 1)
+    extra = None
+    if rank == 0 and N == 1 and not args.no_extra:
+        extra = run_extra_workloads(swaa, torch, inputs, flush_l2, stream, peaks)
 
     # ---------------------------------------------------------------- backward pass of the same layer (outside the timed step)
     backward = None
@@ -372,10 +420,10 @@ def run_ours(args, rank, local_rank, world):
         if world > 1:
             dist.destroy_process_group()
         return
-    avg_pre_ms = t_pre / K
+    avg_pre_ms = t_pre  # median over the timed steps (max over ranks)
     achieved = whole_job_value(prefill_flops, 1, avg_pre_ms * 1e-3) / 1e12  # per GPU; the line reports N x this
-    fa_gbs = fa_bytes / (t_fa / K * 1e-3) / 1e9
-    swa_gbs = swa_bytes / (t_swa / K * 1e-3) / 1e9
+    fa_gbs = fa_bytes / (t_fa * 1e-3) / 1e9
+    swa_gbs = swa_bytes / (t_swa * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": N * achieved, "unit": UNIT, "n_gpus": N, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -383,7 +431,8 @@ def run_ours(args, rank, local_rank, world):
         "config": {"workload": "cfg2 long-context SWA prefill: B=1 L=32768 Hq=32 Hkv=8 D=128 W=2048 n_sink=4 "
                                "(K row 0 shifted); step also runs cfg4 decode B=16 Lcache=65536 FA and SWA(W=4096,n_sink=4)",
                    "l2": "flushed before every kernel: 256 MiB write, then 256 MiB read (clean lines)", "parallelism": f"replicas x{N}",
-                   "value_from": "prefill kernel time inside the step (CUDA events on the launching stream)"},
+                   "value_from": "median over the timed steps of the prefill kernel time inside the step "
+                                 "(CUDA events on the launching stream)"},
         "clocks": clocks,
         "e2e": {"value": N * prefill_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": int(q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": int(out.numel()) * 2,
@@ -392,25 +441,64 @@ def run_ours(args, rank, local_rank, world):
         "roofline": {"kernel": "prefill_kernel<128, 0>", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                      "traffic": PREFILL_DRAM_TRAFFIC_BYTES, "peak_source": peaks["source"] + " burst bf16",
-                     "frac_of_nominal_2250": achieved / 2250.0, "ms_per_launch": avg_pre_ms},
+                     "frac_of_nominal_2250": achieved / 2250.0, "ms_per_launch": avg_pre_ms,
+                     "ms_per_launch_min": st_pre["min"], "ms_per_launch_mean": st_pre["mean"],
+                     "achieved_at_min": prefill_flops / (st_pre["min"] * 1e-3) / 1e12},
         "decode": {
-            "fa": {"gbs": N * fa_gbs, "us_per_launch": 1e3 * t_fa / K, "bytes": fa_bytes,
+            "fa": {"gbs": N * fa_gbs, "us_per_launch": 1e3 * t_fa, "us_per_launch_min": 1e3 * st_fa["min"],
+                   "us_per_launch_mean": 1e3 * st_fa["mean"], "bytes": fa_bytes,
                    "roofline": {"bound": "hbm", "achieved": fa_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                 "frac": fa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": fa_gbs / 8000.0,
                                 "traffic": DECODE_FA_DRAM_TRAFFIC_BYTES},
                    "e2e_gbs": fa_bytes / (e2e_fa_ms * 1e-3) / 1e9},
-            "swa": {"gbs": N * swa_gbs, "us_per_launch": 1e3 * t_swa / K, "bytes": swa_bytes,
+            "swa": {"gbs": N * swa_gbs, "us_per_launch": 1e3 * t_swa, "us_per_launch_min": 1e3 * st_swa["min"],
+                    "us_per_launch_mean": 1e3 * st_swa["mean"], "bytes": swa_bytes,
                     "roofline": {"bound": "hbm", "achieved": swa_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": swa_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": swa_gbs / 8000.0,
                                  "traffic": DECODE_SWA_DRAM_TRAFFIC_BYTES},
                     "e2e_gbs": swa_bytes / (e2e_swa_ms * 1e-3) / 1e9},
         },
         "backward": backward,
+        "extra": extra,
         "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_extra_workloads(swaa, torch, inputs, flush_l2, stream, peaks):
+    """The workloads the timed step does not contain, one flushed launch set each, after the timed steps: workload
+    1 (tiny), workload 5 (varlen), the time against L at fixed W (App. A: O(N * W)), and workload 3, the 36-layer
+    interleaved stack with its mask policy from the layer schedule (per kind and in total; the stack runs for
+    seconds, so its total is set against the sustained bf16 peak)."""
+    extra = {"note": "outside the timed step; median of `launches` launches each, L2 flushed before every launch"}
+    extra["cfg1_tiny"] = time_prefill_case(swaa, torch, flush_l2, stream, peaks, inputs.cfg_tiny(), False, 5)
+    extra["cfg5_varlen"] = time_prefill_case(swaa, torch, flush_l2, stream, peaks, inputs.cfg_varlen(), False, 3)
+    extra["linear_in_L"] = [time_prefill_case(swaa, torch, flush_l2, stream, peaks, inputs.cfg_long(L=L), False, 5)
+                            for L in (8192, 16384, 32768, 65536, 131072)]
+    pol = swaa.SwaaPolicy(n_layers=36, window=4096, n_sink=64, fa_start=3, fa_step=4, fa_decode=True)
+    per_kind, flops = {False: [], True: []}, 0.0
+    tensors = None
+    for layer in range(pol.n_layers):
+        cfg = inputs.cfg_stack_layer(layer)
+        full = swaa.schedule_is_full(pol, layer, 0)
+        del tensors
+        tensors = inputs.make_prefill_inputs(cfg, "cuda")
+        r = time_prefill_case(swaa, torch, flush_l2, stream, peaks, cfg, full, 1, tensors=tensors)
+        per_kind[bool(full)].append(r["ms"])
+        flops += r["effective_tflops"] * r["ms"] * 1e9
+    del tensors
+    total = sum(per_kind[False]) + sum(per_kind[True])
+    tf = flops / (total * 1e-3) / 1e12
+    extra["cfg3_stack"] = {
+        "layers": pol.n_layers, "ms_total": total, "effective_tflops": tf,
+        "frac_of_measured_sustained_peak": tf / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": tf / 2250.0,
+        "swa_layers": len(per_kind[False]), "ms_per_swa_layer": sum(per_kind[False]) / len(per_kind[False]),
+        "ms_swa_layer_min": min(per_kind[False]), "ms_swa_layer_max": max(per_kind[False]),
+        "fa_layers": len(per_kind[True]), "ms_per_fa_layer": sum(per_kind[True]) / len(per_kind[True]),
+        "launches_per_layer": 1}
+    return extra
 
 
 def run_profile_case(case: str):
@@ -472,33 +560,15 @@ def run_sweep():
     flush_rd = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
 
+    def flush_l2():
+        flush.zero_()
+        flush_rd.sum()
+
     def time_case(tag, cfg, is_full, reps=5, tensors=None):
-        q, k, v, cu = tensors if tensors is not None else inputs.make_prefill_inputs(cfg, "cuda")
-        out = torch.empty_like(q)
-        ms = []
-        for r in range(reps + 1):
-            flush.zero_()
-            flush_rd.sum()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            swaa.swaa_prefill(q, k, v, out, cu, max(cfg.seqlens), cfg.window, cfg.n_sink, is_full)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if r > 0:
-                ms.append(a.elapsed_time(b))
-        assert swaa.last_device_status() == 0
-        ms.sort()
-        med = ms[len(ms) // 2]
-        pairs = sum(visible_pairs(L, cfg.window, cfg.n_sink, is_full) for L in cfg.seqlens)
-        flops = 4.0 * cfg.D * cfg.Hq * pairs
-        tf = flops / (med * 1e-3) / 1e12
-        line = {"case": tag, "seqlens": list(cfg.seqlens) if len(cfg.seqlens) > 1 else cfg.seqlens[0], "Hq": cfg.Hq,
-                "Hkv": cfg.Hkv, "D": cfg.D, "window": cfg.window, "n_sink": cfg.n_sink, "is_full": bool(is_full),
-                "ms": med, "ms_min": ms[0], "effective_tflops": tf, "frac_of_measured_peak": tf / peaks["bf16_tflops"],
-                "frac_of_nominal_2250": tf / 2250.0, "us_per_1k_tokens": 1e3 * med / (sum(cfg.seqlens) / 1024.0)}
+        line = {"case": tag}
+        line.update(time_prefill_case(swaa, torch, flush_l2, stream, peaks, cfg, is_full, reps, tensors=tensors))
         print(json.dumps(line), flush=True)
-        del out
-        return med
+        return line["ms"]
 
     # time against L at fixed W (App. A: O(N*W)), then the sink and window variants on workload 2
     for L in (8192, 16384, 32768, 65536, 131072):
@@ -661,6 +731,8 @@ def main():
                     choices=["prefill", "prefill_full", "prefill_tiny", "backward", "decode_fa", "decode_swa",
                              "decode_fa_small", "decode_swa_small"],
                     help="run three launches of one kernel only (for ncu) and exit")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the workloads outside the timed step (workloads 1, 3, 5 and the L sweep)")
     ap.add_argument("--sweep", action="store_true",
                     help="time swaa_prefill on the other workloads and the L / W / n_sink sweeps (one GPU) and exit")
     args = ap.parse_args()

@@ -93,7 +93,7 @@ int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out,
                          void* stream);
 
 /*
- * Backward pass of swaa_prefill under the same mask policy (Sec. 3.3: fine-tuning under SWA uses the mask
+ * Backward pass of swaa_prefill under the same mask policy (Sec. 3.2.2: fine-tuning under SWA uses the mask
  * the model will be served with).  Given the forward inputs, the forward output `out`, its log-sum-exp
  * rows `lse` (as written by swaa_prefill) and the gradient `dout` of the loss with respect to `out`, writes
  * the gradients with respect to q, k and v (dk, dv summed over the query heads of each GQA group).
@@ -104,8 +104,10 @@ int swaa_prefill_chunked(const void* q, const void* k, const void* v, void* out,
  *   workspace         device, at least swaa_prefill_backward_workspace_size(B, T, Hq, Hkv, D, n_sink) bytes,
  *                     256-byte aligned; contents need not be initialised (fp32 accumulators for dq and for the
  *                     dk, dv rows of the sink key tiles, and the row terms dout.out and lse * log2(e))
- * Other arguments and status codes as for swaa_prefill.  fp32 accumulation throughout; P and dS are rounded to
- * bf16 for the tensor-core products, as in the forward pass.
+ * Other arguments and status codes as for swaa_prefill: a sequence longer than max_seqlen (or running past T) is
+ * reported as SWAA_ERR_BAD_SEQLENS through the status word; its dk and dv rows are not written and its dq rows are
+ * zero.  fp32 accumulation throughout; P and dS are rounded to bf16 for the tensor-core products, as in the
+ * forward pass.
  */
 size_t swaa_prefill_backward_workspace_size(int B, int T, int Hq, int Hkv, int D, int n_sink);
 

@@ -1,4 +1,4 @@
-// Backward pass of the prefill attention under the same mask policy (for SWA-aware fine-tuning, Sec. 3.3:
+// Backward pass of the prefill attention under the same mask policy (for SWA-aware fine-tuning, Sec. 3.2.2:
 // the adapted model is trained with the mask it will be served with).
 //
 // Given q, k, v, out, dout and the log-sum-exp rows of the forward pass:
@@ -44,6 +44,7 @@ struct BackwardParams {
     __nv_bfloat16* dv;
     const int32_t* cu_seqlens;
     int B, T, Hq, Hkv, G;
+    int max_seqlen;          // the launch covers sequences up to this length; a longer one is reported and skipped
     int window, n_sink, is_full;
     float scale;
 };
@@ -106,14 +107,14 @@ __global__ void backward_convert_dq_kernel(const float* __restrict__ acc, __nv_b
 // dk, dv rows of the split key tiles = bf16(dkv_accum); one thread per four channels of one (b, row, kv head).
 __global__ void backward_convert_dkv_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dk,
                                             __nv_bfloat16* __restrict__ dv, const int32_t* __restrict__ cu_seqlens, int B,
-                                            int T, int sink_rows, int Hkv, int D) {
+                                            int T, int max_seqlen, int sink_rows, int Hkv, int D) {
     const size_t plane = (size_t)B * sink_rows * Hkv * D;
     const size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (e >= plane) return;
     const size_t row = e / ((size_t)Hkv * D);  // b * sink_rows + j
     const int b = (int)(row / sink_rows), j = (int)(row - (size_t)b * sink_rows);
     const int seq_start = cu_seqlens[b], Lseq = cu_seqlens[b + 1] - seq_start;
-    if (j >= Lseq || seq_start < 0 || seq_start + Lseq > T) return;
+    if (j >= Lseq || Lseq > max_seqlen || seq_start < 0 || seq_start + Lseq > T) return;
     const size_t dst = (size_t)(seq_start + j) * Hkv * D + (e - row * (size_t)Hkv * D);
     const float4 a = *reinterpret_cast<const float4*>(acc + e);
     const float4 c = *reinterpret_cast<const float4*>(acc + plane + e);
@@ -159,8 +160,9 @@ backward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     const int seq_start = p.cu_seqlens[b], Lseq = p.cu_seqlens[b + 1] - seq_start;
     const int j0 = n_tile * BT;
-    if (Lseq <= 0 || j0 >= Lseq || seq_start < 0 || seq_start + Lseq > p.T) {
-        if (tid == 0 && (Lseq < 0 || seq_start < 0 || seq_start + Lseq > p.T)) record_device_error(SWAA_ERR_BAD_SEQLENS);
+    if (Lseq <= 0 || Lseq > p.max_seqlen || j0 >= Lseq || seq_start < 0 || seq_start + Lseq > p.T) {
+        if (tid == 0 && (Lseq < 0 || Lseq > p.max_seqlen || seq_start < 0 || seq_start + Lseq > p.T))
+            record_device_error(SWAA_ERR_BAD_SEQLENS);
         return;
     }
     const bool full = p.is_full != 0;

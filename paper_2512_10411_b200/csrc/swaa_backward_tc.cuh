@@ -1,4 +1,4 @@
-// Backward pass of the prefill attention on the tcgen05 tensor cores (head dimension 128), Sec. 3.3.
+// Backward pass of the prefill attention on the tcgen05 tensor cores (head dimension 128), Sec. 3.2.2.
 //
 // One block owns a tile of 128 keys of one (sequence, kv head) and walks the 64-row query tiles that can
 // see it, for every query head of the GQA group.  All five products of a step run as tcgen05.mma with the
@@ -114,8 +114,9 @@ backward_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
     const int seq_start = p.cu_seqlens[b], Lseq = p.cu_seqlens[b + 1] - seq_start;
     const int j0 = n_tile * BK;
-    if (Lseq <= 0 || j0 >= Lseq || seq_start < 0 || seq_start + Lseq > p.T) {  // uniform: before any barrier or allocation
-        if (threadIdx.x == 0 && (Lseq < 0 || seq_start < 0 || seq_start + Lseq > p.T))
+    if (Lseq <= 0 || Lseq > p.max_seqlen || j0 >= Lseq || seq_start < 0 ||
+        seq_start + Lseq > p.T) {  // uniform: before any barrier or allocation
+        if (threadIdx.x == 0 && (Lseq < 0 || Lseq > p.max_seqlen || seq_start < 0 || seq_start + Lseq > p.T))
             record_device_error(SWAA_ERR_BAD_SEQLENS);
         return;
     }

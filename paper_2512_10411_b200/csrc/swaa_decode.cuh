@@ -152,14 +152,6 @@ __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumerThreads) : "memory");
 }
 
-#ifdef SWAA_DECODE_TIMING
-// Development aid: per-block time stamps (ns) of the phases of one launch.
-__device__ unsigned long long g_decode_stamps[256][8];
-#define SWAA_DSTAMP(slot) do { if ((threadIdx.x & 31) == 0 && blockIdx.x < 256) g_decode_stamps[blockIdx.x][slot] = global_timer_ns(); } while (0)
-#else
-#define SWAA_DSTAMP(slot)
-#endif
-
 template <int D, int NH, bool kPaged>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -188,12 +180,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     __shared__ int sc_b0;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef SWAA_DECODE_REVERSE_BLOCKS  // development aid: hand the runs of the tile list out in reverse block order
-    const int ncta = (int)gridDim.x, cta = (int)(gridDim.x - 1 - blockIdx.x);
-#else
     const int ncta = (int)gridDim.x, cta = (int)blockIdx.x;
-#endif
-    if (warp == 0) SWAA_DSTAMP(0);  // block entered
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -305,7 +292,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         off0 = sc_off;
     }
     if (t0 >= t1) return;  // nothing for this block (uniform; nobody waits on a barrier)
-    if (warp == 0) SWAA_DSTAMP(1);  // start position known
     const int cnt = (int)(t1 - t0);  // tpc <= tiles of the whole problem / blocks, far below 2^31 in practice
 
     if (warp == kDecodeConsumerWarps) {
@@ -415,8 +401,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             const int vw = w.vend() - 16 * warp;            // this warp's keys [vb, vw) of its 16 are visible
             const int vb = kPaged ? max(w.vbegin() - 16 * warp, 0) : 0;
             const uint32_t stage = smem_base + (uint32_t)s * L::kStageBytes;
-            ok = ok && mbar_wait(bar_kf(s), ph, abort_flag);
-            if (warp == 0 && n == 0) SWAA_DSTAMP(2);  // first K tile landed
+            // warp-wide decisions after a bounded wait: ldmatrix, mma.sync and the shuffles need all 32 lanes
+            ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_kf(s), ph, abort_flag));
             if (ok && min(vw, 16) > vb) {  // some of this warp's 16 keys are visible
                 // ---- S^T = K Q^T : rows = keys (g, g+8), cols = heads (2c, 2c+1)
                 float sacc[NH][4];
@@ -472,7 +458,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
 
                 // ---- O^T += V^T P^T : rows = channels (16qb + g, 16qb + g + 8), cols = heads (2c, 2c+1)
-                ok = mbar_wait(bar_vf(s), ph, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_vf(s), ph, abort_flag));
                 if (ok) {
                     // rows of the tile past the last visible key may hold anything (also NaN): clear them
                     auto vis = [&](int key) { return key < vw && key >= vb; };
@@ -496,7 +482,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     }
                 }
             } else {
-                ok = ok && mbar_wait(bar_vf(s), ph, abort_flag);
+                ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_vf(s), ph, abort_flag));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_e(s));
@@ -507,7 +493,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
 
         // ---- merge the four warps of the block through shared memory
-        if (warp == 0 && n == cnt) SWAA_DSTAMP(3);  // last tile consumed
 #pragma unroll
         for (int nh = 0; nh < NH; ++nh) {
 #pragma unroll
@@ -631,7 +616,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         consumer_sync();  // the merge buffers are free for the next segment
         first_seg = false;
     }
-    if (warp == 0) SWAA_DSTAMP(4);  // done
 }
 
 }  // namespace swaa

@@ -384,6 +384,9 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
     if (ub > 2147483647LL / p.n_pairs) return SWAA_ERR_UNSUPPORTED;
     p.tiles_ub = (int)ub;
     if (p.tiles_ub == 0) return SWAA_OK;  // max_seqlen == 0: nothing can be valid
+    // a window that covers the longest key sequence is full causal attention for every row; clamping keeps the
+    // kernel's 32-bit column arithmetic (column - window) far from overflow
+    if (!is_full && max_seqlen_k >= 1 && window > max_seqlen_k) window = max_seqlen_k;
     p.window = window;
     p.n_sink = n_sink;
     p.is_full = is_full ? 1 : 0;
@@ -501,7 +504,7 @@ static int launch_backward(const void* q, const void* k, const void* v, const vo
         const int sink_rows = p.sink_tiles * kKeyTile;
         const size_t plane = (size_t)p.B * sink_rows * p.Hkv * D;
         backward_convert_dkv_kernel<<<(unsigned)((plane / 4 + 255) / 256), 256, 0, st>>>(
-            p.dkv_accum, p.dk, p.dv, p.cu_seqlens, p.B, p.T, sink_rows, p.Hkv, D);
+            p.dkv_accum, p.dk, p.dv, p.cu_seqlens, p.B, p.T, p.max_seqlen, sink_rows, p.Hkv, D);
         ++launches;
     }
     launch_counter().fetch_add((uint64_t)launches, std::memory_order_relaxed);
@@ -550,6 +553,7 @@ extern "C" int swaa_prefill_backward(const void* q, const void* k, const void* v
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.G = Hq / Hkv;
+    p.max_seqlen = max_seqlen;
     p.window = window;
     p.n_sink = n_sink;
     p.is_full = is_full ? 1 : 0;
@@ -748,25 +752,5 @@ extern "C" int swaa_last_device_status(void* stream) {
     }
     return value;
 }
-
-#ifdef SWAA_DECODE_TIMING
-extern "C" int swaa_debug_read_decode_stamps(unsigned long long* out, int n_blocks) {
-    if (n_blocks > 256) n_blocks = 256;
-    if (cudaMemcpyFromSymbol(out, g_decode_stamps, sizeof(unsigned long long) * 8 * n_blocks) != cudaSuccess)
-        return SWAA_ERR_CUDA;
-    return SWAA_OK;
-}
-#endif
-
-#ifdef SWAA_PHASE_TIMING
-extern "C" int swaa_debug_read_phases(unsigned long long* out32, int reset) {
-    if (cudaMemcpyFromSymbol(out32, g_phase_cycles, sizeof(unsigned long long) * 32) != cudaSuccess) return SWAA_ERR_CUDA;
-    if (reset) {
-        unsigned long long z[32] = {0};
-        if (cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z)) != cudaSuccess) return SWAA_ERR_CUDA;
-    }
-    return SWAA_OK;
-}
-#endif
 
 extern "C" uint64_t swaa_kernel_launch_count(void) { return launch_counter().load(std::memory_order_relaxed); }

@@ -131,9 +131,11 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 }
 
 // 2^x for a pair of arguments on the FMA and integer pipes instead of the special-function unit:
-// x = n + f with n = round(x), f in [-1/2, 1/2]; 2^f by a cubic (relative error 7.6e-5, far below the
-// bf16 rounding of P); n is added into the exponent field.  Arguments below -126 (masked scores arrive
-// as -inf) give exactly 0, as ex2.approx.ftz does.
+// x = n + f with n = round(x), f in [-1/2, 1/2]; 2^f by a cubic with constant term exactly 1 (minimax fit of
+// the other three coefficients: relative error 1.0e-4, far below the bf16 rounding of P), so that 2^0 = 1
+// exactly as on the special-function unit and a row of equal scores sums to its key count; n is added into
+// the exponent field.  Arguments below -126 (masked scores arrive as -inf) give exactly 0, as
+// ex2.approx.ftz does.
 __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, float& r1) {
     const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
     const uint64_t xx = pack_f32x2(x0, x1);
@@ -141,10 +143,10 @@ __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, floa
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(t) : "l"(xx), "l"(pack_f32x2(kMagic, kMagic)));
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(fl) : "l"(t), "l"(pack_f32x2(kMagic, kMagic)));
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(f) : "l"(xx), "l"(fl));
-    q = fma_f32x2(f, pack_f32x2(0.05520550534129143f, 0.05520550534129143f),
-                  pack_f32x2(0.24261397123336792f, 0.24261397123336792f));
-    q = fma_f32x2(q, f, pack_f32x2(0.6932547688484192f, 0.6932547688484192f));
-    q = fma_f32x2(q, f, pack_f32x2(0.9999276995658875f, 0.9999276995658875f));
+    q = fma_f32x2(f, pack_f32x2(0.055009059607982635f, 0.055009059607982635f),
+                  pack_f32x2(0.2422109693288803f, 0.2422109693288803f));
+    q = fma_f32x2(q, f, pack_f32x2(0.6932829022407532f, 0.6932829022407532f));
+    q = fma_f32x2(q, f, pack_f32x2(1.0f, 1.0f));
     float t0, t1, q0, q1;
     unpack_f32x2(t, t0, t1);
     unpack_f32x2(q, q0, q1);
@@ -153,10 +155,7 @@ __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, floa
 }
 
 // Bit c (0..15) set: column pair c of every 32-column chunk of a score tile takes the polynomial path.
-#ifndef SWAA_POLY_PAIR_MASK
-#define SWAA_POLY_PAIR_MASK 0x8080u
-#endif
-constexpr uint32_t kPolyPairMask = SWAA_POLY_PAIR_MASK;
+constexpr uint32_t kPolyPairMask = 0x8080u;
 
 #define SWAA_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
 #define SWAA_I8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
@@ -206,17 +205,6 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int b_mn_major) 
            ((uint32_t)(M >> 4) << 24);
 }
 
-#ifdef SWAA_PHASE_TIMING
-// Development aid: per-phase cycle sums of the softmax role (side A: 0-7, side B: 8-15) and of the
-// issuer's waits (16-23), accumulated over all blocks.
-__device__ unsigned long long g_phase_cycles[32];
-#define SWAA_TICK(var) const long long var = clock64()
-#define SWAA_PHASE_ADD(slot, cycles) atomicAdd(&g_phase_cycles[slot], (unsigned long long)(cycles))
-#else
-#define SWAA_TICK(var)
-#define SWAA_PHASE_ADD(slot, cycles)
-#endif
-
 template <int D>
 struct PrefillSmem {
     static constexpr int kTileBytes = 128 * D * 2;  // one 128-row tile of Q, K or V
@@ -229,8 +217,8 @@ struct PrefillSmem {
     static constexpr int kOffStage = kOffV + kStages * kTileBytes;  // 8 x 4 KiB: per-warp output staging
     static constexpr int kOffBar = kOffStage + 8 * 4096;
     // barriers: Q full/empty, K full/empty, V full/empty per stage, per side S-full / P-ready / O-done /
-    // O-free, work-descriptor full/empty per slot, final
-    static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1 + 1;
+    // O-free, work-descriptor full/empty per slot, final, V-tile-cleared per stage (paged keys only)
+    static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1 + kStages;
     static constexpr int kOffMisc = kOffBar + kNumBars * 8;      // tmem slot, abort flag, work descriptors
     static constexpr int kBytes = kOffMisc + 128;
     static constexpr int kDynamicBytes = kBytes + 1024;          // room to align the base to 1024 B
@@ -269,8 +257,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     constexpr int BAR_QF = 0, BAR_QE = 1, BAR_KF = 2, BAR_KE = BAR_KF + ST, BAR_VF = BAR_KE + ST, BAR_VE = BAR_VF + ST;
     constexpr int BAR_SF = BAR_VE + ST, BAR_PR = BAR_SF + 2, BAR_OD = BAR_PR + 2, BAR_OF = BAR_OD + 2;
     constexpr int BAR_WF = BAR_OF + 2, BAR_WE = BAR_WF + 2, BAR_FIN = BAR_WE + 2;
-    constexpr int BAR_VC = BAR_FIN + 1;  // paged only: the rows of a V tile past the last key have been cleared
-    static_assert(BAR_VC + 1 == L::kNumBars, "barrier count");
+    // paged only, one per ring stage: the rows of the V tile in that stage past the last key have been cleared.
+    // Completed once per cleared tile; producer and issuer each keep the stage's phase bit.  The producer cannot
+    // clear a stage twice before the issuer has waited for the first clear: reusing the stage needs the
+    // issuer's V-empty commit, which follows that wait.
+    constexpr int BAR_VC = BAR_FIN + 1;
+    static_assert(BAR_VC + ST == L::kNumBars, "barrier count");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + L::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* work_ring = reinterpret_cast<volatile int*>(tmem_slot + 4);  // 2 slots x 8 ints
@@ -459,7 +451,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                                     for (int j = 0; j < 8; ++j)
                                         st_shared_v4(sV + s * L::kTileBytes + pn * L::kPanelBytes + r * 128 + j * 16, 0u, 0u, 0u, 0u);
                             fence_proxy_async_smem();
-                            mbar_arrive(bar(BAR_VC));
+                            mbar_arrive(bar(BAR_VC + s));
                         }
                     }
                 }
@@ -522,7 +514,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             int gs[2] = {0, 0};        // tiles processed per side (phase of S-full / P-ready / O-done)
             int items_side[2] = {0, 0};
             int items = 0;
-            int n_cleared = 0;  // V tiles whose rows past the sequence end were cleared (paged only)
+            uint32_t vc_phase = 0;  // paged only: bit s = phase of the stage's V-tile-cleared barrier
             bool ok = true;
             for (int it = 0; ok; ++it) {
                 WorkItem w;
@@ -560,8 +552,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                          mbar_wait(bar(BAR_PR + 0), (uint32_t)gs[0] & 1u, abort_flag);
                     if (kPaged && ok && w.k_off + w.seq_len - trng.tile(n) * BN < BN) {
                         // last key tile of a sequence that ends inside it: the producer clears the rows past the end
-                        ok = mbar_wait(bar(BAR_VC), (uint32_t)n_cleared & 1u, abort_flag);
-                        ++n_cleared;
+                        ok = mbar_wait(bar(BAR_VC + sv), (vc_phase >> sv) & 1u, abort_flag);
+                        vc_phase ^= 1u << sv;
                     }
                     // the first PV of an item overwrites O: the previous item's epilogue must have read it
                     if (ok && n == 0) ok = mbar_wait(bar(BAR_OF + 0), ((uint32_t)items_side[0] & 1u) ^ 1u, abort_flag);
@@ -621,7 +613,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         bool ok = true;
         for (int it = 0; ok; ++it) {
             WorkItem w;
-            ok = fetch_work(it, w, false);
+            // every decision taken after a bounded wait is made for the whole warp: the warp-wide tensor-memory
+            // instructions and votes below need all 32 lanes
+            ok = __all_sync(0xffffffffu, fetch_work(it, w, false));
             if (!ok) break;
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_WE + (it & 1)));
@@ -642,18 +636,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (int n = 0; n < nt; ++n, ++gs) {
                 const int j0 = tr.tile(n) * BN;
                 const bool need_mask = tile_needs_mask(i0, i1, j0, j0 + BN - 1, p.window, p.n_sink, full);
-                SWAA_TICK(c0);
-                ok = mbar_wait(bar(BAR_SF + side), (uint32_t)gs & 1u, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SF + side), (uint32_t)gs & 1u, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
-                SWAA_TICK(c1);
                 uint32_t sr[128];
                 tmem_ld32(tS + 0, sr + 0);
                 tmem_ld32(tS + 32, sr + 32);
                 tmem_ld32(tS + 64, sr + 64);
                 tmem_ld32(tS + 96, sr + 96);
                 tc_wait_ld();
-                SWAA_TICK(c2);
                 uint32_t vis[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
                 if (need_mask) {
                     // Bit b of vis[cc] <=> column c = 32*cc + b of this tile is visible to this row:
@@ -703,7 +694,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 } else if (m_used == -INFINITY) {
                     m_used = m_new;  // nothing accumulated yet for this row
                 }
-                SWAA_TICK(c3);
                 const float off = (m_used == -INFINITY) ? 0.f : m_used * p.sl2;
                 const uint64_t sl2x2 = pack_f32x2(p.sl2, p.sl2), noffx2 = pack_f32x2(-off, -off);
                 uint64_t psum_a = pack_f32x2(0.f, 0.f), psum_b = pack_f32x2(0.f, 0.f);
@@ -742,26 +732,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     unpack_f32x2(add_f32x2(psum_a, psum_b), a0, a1);
                     l_sum += a0 + a1;
                 }
-                SWAA_TICK(c4);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(BAR_PR + side));
-#ifdef SWAA_PHASE_TIMING
-                if (lane == 0 && wq == 0) {
-                    const long long c5 = clock64();
-                    SWAA_PHASE_ADD(side * 8 + 0, c1 - c0);  // wait for S
-                    SWAA_PHASE_ADD(side * 8 + 1, c2 - c1);  // TMEM load
-                    SWAA_PHASE_ADD(side * 8 + 2, c3 - c2);  // mask + max (+ rescale)
-                    SWAA_PHASE_ADD(side * 8 + 3, c4 - c3);  // exp, pack, store issue
-                    SWAA_PHASE_ADD(side * 8 + 4, c5 - c4);  // store wait + arrive
-                    SWAA_PHASE_ADD(side * 8 + 5, 1);        // tiles
-                }
-#endif
             }
             if (!ok) break;
             // ---- epilogue of this item: O / l -> bf16 -> global
-            SWAA_TICK(e0);
-            ok = mbar_wait(bar(BAR_OD + side), (uint32_t)items_done & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OD + side), (uint32_t)items_done & 1u, abort_flag));
             if (!ok) break;
             ++items_done;
             tc_fence_after();
@@ -771,7 +748,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             tc_wait_ld();
             tc_fence_before();
             mbar_arrive(bar(BAR_OF + side));  // O may be overwritten by the next item's first PV
-            SWAA_TICK(e1);
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             if (q0 + wq * 32 + 31 < seq_len) {
                 // all 32 rows of this warp are valid: stage [32 rows][64 ch] panels in shared memory in the
@@ -814,14 +790,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const float lse2 = (m_used == -INFINITY) ? -INFINITY : m_used * p.sl2 + log2f(l_sum);
                 p.lse[(size_t)h * p.T + seq_start + iq] = lse2 * 0.6931471805599453f;
             }
-#ifdef SWAA_PHASE_TIMING
-            if (lane == 0 && wq == 0) {
-                const long long e2 = clock64();
-                SWAA_PHASE_ADD(side * 8 + 6, e1 - e0);  // epilogue: wait + O load
-                SWAA_PHASE_ADD(side * 8 + 7, e2 - e1);  // epilogue: convert + store
-                SWAA_PHASE_ADD(16 + side, 1);           // items
-            }
-#endif
         }
         if (lane == 0) tma_store_wait_all();  // outstanding output stores of this warp
     }

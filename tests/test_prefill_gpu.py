@@ -215,10 +215,61 @@ def test_prefill_varlen_workload():
     sampled_check(inputs.cfg_varlen(), 2048)
 
 
-@pytest.mark.parametrize("layer", [0, 3])
+@pytest.mark.parametrize("layer", [0, 3, 4, 7, 35])
 def test_prefill_stack_layer(layer):
-    """Workload 3: one SWA layer (0) and one FA layer (3) of the 36-layer stack at L=131072."""
+    """Workload 3: SWA layers (0, 4) and FA layers (3, 7, 35) of the 36-layer stack at L=131072."""
     pol = swaa.SwaaPolicy(36, 4096, 64, 3, 4, False)
     full = swaa.schedule_is_full(pol, layer, 0)
     assert full == (layer % 4 == 3)
     sampled_check(inputs.cfg_stack_layer(layer), 2048 if not full else 512, is_full=full)
+
+
+def closed_form_counts(seqlens, W, S, full):
+    """Visible keys of every packed row: i + 1 under full attention, else the window part min(i + 1, W) plus the
+    sink keys that lie before the window, max(0, min(S, i - W + 1))."""
+    parts = []
+    for n in seqlens:
+        i = np.arange(n, dtype=np.int64)
+        parts.append(i + 1 if full else np.minimum(i + 1, W) + np.clip(i - W + 1, 0, S))
+    return np.concatenate(parts)
+
+
+BIG_COUNT_CASES = {
+    "cfg2_swa": (lambda: inputs.cfg_long(), False),
+    "cfg2_full": (lambda: inputs.cfg_long(is_full=True), True),
+    "cfg3_layer0_swa": (lambda: inputs.cfg_stack_layer(0), False),
+    "cfg3_layer3_full": (lambda: inputs.cfg_stack_layer(3), True),
+    "cfg5_varlen": (lambda: inputs.cfg_varlen(), False),
+}
+
+
+@pytest.mark.parametrize("case", sorted(BIG_COUNT_CASES))
+def test_prefill_every_row_sees_the_right_number_of_keys_at_full_size(case):
+    """Q = 0 makes every visible score equal, so exp(lse) of a row is the number of keys it saw: one launch per
+    full-size workload checks that count for EVERY (row, head) against the closed form, which is itself checked
+    against the oracle's enumeration on boundary rows and a seeded sample."""
+    make, full = BIG_COUNT_CASES[case]
+    cfg = make()
+    T = cfg.T
+    g = torch.Generator(device="cuda").manual_seed(cfg.seed)
+    q = torch.zeros((T, cfg.Hq, cfg.D), dtype=torch.bfloat16, device="cuda")
+    k = torch.randn((T, cfg.Hkv, cfg.D), generator=g, device="cuda").to(torch.bfloat16)
+    v = torch.ones((T, cfg.Hkv, cfg.D), dtype=torch.bfloat16, device="cuda")
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(cfg.seqlens)]).astype(np.int32), device="cuda")
+    out = torch.empty_like(q)
+    lse = torch.full((cfg.Hq, T), float("nan"), dtype=torch.float32, device="cuda")
+    swaa.swaa_prefill(q, k, v, out, cu, max(cfg.seqlens), cfg.window, cfg.n_sink, full, lse=lse)
+    assert swaa.last_device_status() == 0
+    want = closed_form_counts(cfg.seqlens, cfg.window, cfg.n_sink, full)
+    got = torch.exp(lse.double())
+    want_t = torch.from_numpy(want).cuda().double()
+    dev = (got - want_t[None, :]).abs().max().item()
+    assert torch.equal(torch.round(got), want_t[None, :].expand_as(got)), f"{case}: largest deviation {dev}"
+    assert (out == 1).all(), "uniform softmax over all-ones values"
+    # the closed form against the oracle's own enumeration
+    rt, rh = sampled_rows(cfg, 256, seed=cfg.seed)
+    qh = np.zeros((T, cfg.Hq, 1), dtype=np.float32)
+    kh = np.zeros((T, cfg.Hkv, 1), dtype=np.float32)
+    ref = oracle.prefill(qh, kh, kh, cu.cpu().numpy(), cfg.window, cfg.n_sink, full, rows=(rt, rh))
+    assert np.array_equal(ref["nvis"], want[rt])
+    print(f"{case}: every one of {T * cfg.Hq} rows counted; largest |exp(lse) - count| = {dev:.3g}")

@@ -94,6 +94,25 @@ def test_paged_prefill_long_context_sampled_rows():
     assert not torch.isnan(out.float()).any()
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_paged_prefill_many_short_sequences_walk_single_tile_ragged_items(D):
+    """Many sequences of fewer than 128 keys with several head pairs per kv head: every block walks a run of items
+    whose only key tile is ragged, so consecutive tiles in different ring stages each need their rows past the
+    sequence end cleared before the product may read them (one cleared-barrier per stage)."""
+    rng = np.random.default_rng(17)
+    B, Hq, Hkv, page = 96, 8, 2, 128
+    lk = tuple(int(x) for x in rng.integers(1, 128, B))
+    lq = tuple(int(rng.integers(1, n + 1)) for n in lk)
+    q, kp, vp, cu_q, sk, bt = make_paged(lq, lk, Hq, Hkv, D, page, seed=811 + D)
+    qh, kh, vh = (inputs.to_f32_numpy(t) for t in (q, kp, vp))
+    for W, S, full in ((1, 0, True), (40, 3, False)):
+        for _ in range(3):  # the hazard was a matter of timing: run it a few times
+            out, lse, status = run_paged(q, kp, vp, cu_q, sk, bt, max(lq), W, S, full)
+            assert status == 0
+        ref = oracle.prefill_paged(qh, kh, vh, cu_q.cpu().numpy(), lk, bt.cpu().numpy(), W, S, full)
+        check_against_oracle(out, ref["out"], f"many short paged sequences D={D} full={full}")
+
+
 def test_paged_prefill_reports_a_bad_page_index():
     q, kp, vp, cu_q, sk, bt = make_paged((10, 20), (200, 20), 2, 1, 64, 128, seed=9, poison=False)
     bt2 = bt.clone()

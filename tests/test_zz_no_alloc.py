@@ -5,14 +5,18 @@ path, a plug-in without access to the host framework's memory pool, a process wh
 fully handed out).  For them the library carries its split-K scratch in a fixed 2 MiB array of its own.
 This test calls that entry point through the C ABI twice in a row, with different shapes and masks so
 that the second call finds the first call's leftovers in the shared array, and checks each result
-against swaa_decode with a caller-owned workspace.  It is collected last on purpose.
+against swaa_decode with a caller-owned workspace and against the float64 oracle.  It also watches the
+driver's free-memory figure and the library's launch counter across each call: nothing may be
+allocated and nothing but the one decode kernel may be launched (no clearing of the scratch).  It is
+collected last on purpose.
 """
 import pytest
 import torch
 
+import oracle
 import paper_2512_10411_b200 as swaa
 from paper_2512_10411_b200 import inputs
-from helpers import ABS_TOL, REL_TOL
+from helpers import ABS_TOL, REL_TOL, check_against_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -44,11 +48,21 @@ def test_decode_static_matches_decode_on_two_calls_in_a_row():
         assert swaa.decode_num_blocks(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.Lmax, W, S, full) > 1
         want = _reference(q, kc, vc, sl, W, S, full)
         got = torch.full_like(q, float("nan"))
-        before = torch.cuda.memory_allocated()
+        torch.cuda.synchronize()
+        # torch's own counter only sees torch's allocator; the driver's free-memory figure also sees a cudaMalloc
+        # made inside the library.  (The very first call in a process may load the module: it is made above, by
+        # _reference, through the same kernel.)
+        torch_before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+        launches_before = swaa.kernel_launch_count()
         swaa.swaa_decode_static(q, kc, vc, got, sl, W, S, full)
-        assert torch.cuda.memory_allocated() == before
+        assert swaa.kernel_launch_count() - launches_before == 1, "one decode kernel, no clearing launch"
         assert swaa.last_device_status() == 0
+        assert torch.cuda.memory_allocated() == torch_before
+        assert torch.cuda.mem_get_info()[0] >= free_before, "device memory was taken during the call"
         assert _close(got, want), cfg.name
+        ref = oracle.decode(inputs.to_f32_numpy(q), inputs.to_f32_numpy(kc), inputs.to_f32_numpy(vc),
+                            sl.cpu().numpy(), W, S, full)
+        check_against_oracle(got, ref["out"], f"decode_static {cfg.name}")
 
 
 def test_decode_static_rejects_shapes_beyond_its_scratch():
