@@ -364,10 +364,6 @@ def run_ours(args, rank, local_rank, world):
         [total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms], world, dev)
     K, N = args.steps, world
 
-    # ---------------------------------------------------------------- the other workloads and the L sweep (N = 1)
-    extra = None
-    if rank == 0 and N == 1 and not args.no_extra:
-        extra = run_extra_workloads(swaa, torch, inputs, flush_l2, stream, peaks)
 
     # ---------------------------------------------------------------- backward pass of the same layer (outside the timed step)
     backward = None
@@ -395,6 +391,11 @@ def run_ours(args, rank, local_rank, world):
         backward = {"ms": bms[len(bms) // 2], "effective_tflops": btf, "frac_of_measured_peak": btf / peaks["bf16_tflops"],
                     "note": "swaa_prefill_backward on the same workload, whole call, median of 5, L2 flushed; not part of the step"}
         del lse, grad_out, dq_, dk_, dv_, bws
+
+    # ---------------------------------------------------------------- the other workloads and the L sweep (N = 1)
+    extra = None
+    if rank == 0 and N == 1 and not args.no_extra:
+        extra = run_extra_workloads(swaa, torch, inputs, flush_l2, stream, peaks)
 
     cpu_baseline = None
     if rank == 0 and N == 1:

@@ -9,8 +9,12 @@ from .swaa_oracle import (  # noqa: F401
     build,
     count_pairs,
     decode,
+    decode_combine,
+    decode_partial,
     decode_paged,
     layer_is_full,
+    layer_is_full_mask,
+    select_fa_layers,
     lazy_ratio,
     num_threads,
     prefill,
@@ -18,6 +22,7 @@ from .swaa_oracle import (  # noqa: F401
     prefill_backward_c,
     prefill_backward_rows,
     prefill_chunked,
+    prefill_cp,
     prefill_paged,
     visible,
 )

@@ -167,14 +167,18 @@ int swaa_oracle_prefill(const float* q, const float* k, const float* v, const in
  * len_k - len_q + i of its sequence and sees the keys the mask policy allows for that position.
  *   q [Tq, Hq, D] packed by cu_q [B+1]; k, v [Tk, Hkv, D] packed by cu_k [B+1]; float32 (bf16 values).
  * Rows are chosen as in swaa_oracle_prefill, row_t being a packed QUERY token index.
+ * is_full_seq (nullable, [B]): a mask policy per sequence, for a batch that mixes sequences in different phases
+ * (Fig. 1a: prefill tokens under the SWA mask next to generated tokens under full attention); when given it
+ * replaces is_full, sequence b being full causal iff is_full_seq[b] != 0.
  * Returns 0, or -1 on inconsistent arguments (also len_q > len_k).
  */
 int swaa_oracle_prefill_chunked(const float* q, const float* k, const float* v, const int32_t* cu_q,
                                 const int32_t* cu_k, int B, int Hq, int Hkv, int D, int64_t W, int64_t S,
-                                int is_full, double scale, int64_t n_rows, const int64_t* row_t,
-                                const int32_t* row_h, double* out, double* lse, double* psum, int64_t* nvis) {
+                                int is_full, const uint8_t* is_full_seq, double scale, int64_t n_rows,
+                                const int64_t* row_t, const int32_t* row_h, double* out, double* lse, double* psum,
+                                int64_t* nvis) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0) return -1;
-    if (!is_full && W < 1) return -1;
+    if ((!is_full || is_full_seq) && W < 1) return -1;
     if (S < 0) return -1;
     const int G = Hq / Hkv;
     const int64_t Tq = B > 0 ? cu_q[B] : 0;
@@ -204,8 +208,9 @@ int swaa_oracle_prefill_chunked(const float* q, const float* k, const float* v, 
             int64_t i = (lk - lq) + (t - cu_q[b]); /* position of the query inside its sequence */
             int64_t kstart = cu_k[b];
             int hk = h / G;
+            const int full_b = is_full_seq ? (is_full_seq[b] != 0) : is_full;
             oracle_row(q + (t * Hq + h) * (int64_t)D, k + (kstart * Hkv + hk) * (int64_t)D,
-                       v + (kstart * Hkv + hk) * (int64_t)D, i, (int64_t)Hkv * D, D, W, S, is_full, scale,
+                       v + (kstart * Hkv + hk) * (int64_t)D, i, (int64_t)Hkv * D, D, W, S, full_b, scale,
                        out + r * D, lse ? lse + r : NULL, psum ? psum + r : NULL, nvis ? nvis + r : NULL, scores);
         }
         free(scores);
@@ -243,6 +248,180 @@ int swaa_oracle_decode(const float* q, const float* kcache, const float* vcache,
         free(scores);
     }
     return 0;
+}
+
+/*
+ * Decode with the cache of every sequence cut along the context (App. A: the full-context cache must be retained
+ * under FA decode, which is what makes splitting it over several devices attractive).  One shard holds the
+ * entries at positions [pos0, pos0 + Lshard) of every sequence: kshard, vshard [B, Lshard, Hkv, D], entry p at row
+ * p - pos0.  seqlens [B] are the TOTAL lengths; the query sits at position seqlens[b] - 1 and sees the keys the
+ * mask policy allows for that position (Sec. 3.1.1, 3.2.1), of which this shard contributes those it holds.
+ * part [B, Hq, D + 2] double: (m, l, o[D]) with m = max of the visible scores of the shard, l = sum exp(s - m),
+ * o = sum exp(s - m) v.  A shard that holds no visible key of a row gives (-inf, 0, 0...).  nvis [B, Hq] (nullable).
+ */
+int swaa_oracle_decode_partial(const float* q, const float* kshard, const float* vshard, const int32_t* seqlens, int B,
+                               int64_t Lshard, int64_t pos0, int Hq, int Hkv, int D, int64_t W, int64_t S,
+                               int is_full, double scale, double* part, int64_t* nvis) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0 || Lshard < 0 || pos0 < 0) return -1;
+    if (!is_full && W < 1) return -1;
+    if (S < 0) return -1;
+    const int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b)
+        if (seqlens[b] < 1) return -1;
+#pragma omp parallel
+    {
+        double* scores = (double*)malloc(sizeof(double) * (size_t)(Lshard > 0 ? Lshard : 1));
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t r = 0; r < (int64_t)B * Hq; ++r) {
+            const int b = (int)(r / Hq), h = (int)(r % Hq), hk = h / G;
+            const int64_t i = (int64_t)seqlens[b] - 1;
+            const float* qi = q + r * D;
+            double* pr = part + r * (D + 2);
+            double m = -INFINITY;
+            int64_t cnt = 0;
+            for (int64_t jl = 0; jl < Lshard; ++jl) {
+                if (!swaa_oracle_visible(i, pos0 + jl, W, S, is_full)) continue;
+                const float* kj = kshard + (((int64_t)b * Lshard + jl) * Hkv + hk) * D;
+                double sdot = 0.0;
+                for (int d = 0; d < D; ++d) sdot += (double)qi[d] * (double)kj[d];
+                scores[jl] = sdot * scale;
+                if (scores[jl] > m) m = scores[jl];
+                ++cnt;
+            }
+            double l = 0.0;
+            for (int d = 0; d < D; ++d) pr[2 + d] = 0.0;
+            for (int64_t jl = 0; jl < Lshard; ++jl) {
+                if (!swaa_oracle_visible(i, pos0 + jl, W, S, is_full)) continue;
+                const double e = exp(scores[jl] - m);
+                const float* vj = vshard + (((int64_t)b * Lshard + jl) * Hkv + hk) * D;
+                l += e;
+                for (int d = 0; d < D; ++d) pr[2 + d] += e * (double)vj[d];
+            }
+            pr[0] = m;
+            pr[1] = l;
+            if (nvis) nvis[r] = cnt;
+        }
+        free(scores);
+    }
+    return 0;
+}
+
+/*
+ * Log-sum-exp combine of P partial results per row (the cross-split merge of a split-K decode, here across
+ * shards): M = max_s m_s, out = sum_s e^(m_s - M) o_s / sum_s e^(m_s - M) l_s; shards with l_s = 0 are skipped;
+ * a row for which every shard is empty gives zeros.  part [P, n_rows, D + 2], out [n_rows, D].
+ */
+int swaa_oracle_decode_combine(const double* part, int P, int64_t n_rows, int D, double* out) {
+    if (P < 1 || n_rows < 0 || D <= 0) return -1;
+    for (int64_t r = 0; r < n_rows; ++r) {
+        double M = -INFINITY;
+        for (int s = 0; s < P; ++s) {
+            const double* pr = part + ((int64_t)s * n_rows + r) * (D + 2);
+            if (pr[1] > 0.0 && pr[0] > M) M = pr[0];
+        }
+        double den = 0.0;
+        for (int d = 0; d < D; ++d) out[r * D + d] = 0.0;
+        for (int s = 0; s < P; ++s) {
+            const double* pr = part + ((int64_t)s * n_rows + r) * (D + 2);
+            if (!(pr[1] > 0.0)) continue;
+            const double w = exp(pr[0] - M);
+            den += w * pr[1];
+            for (int d = 0; d < D; ++d) out[r * D + d] += w * pr[2 + d];
+        }
+        if (den > 0.0)
+            for (int d = 0; d < D; ++d) out[r * D + d] /= den;
+    }
+    return 0;
+}
+
+/*
+ * Context-parallel prefill: one participant owns a contiguous stretch of every sequence (App. A: SWA prefill is
+ * O(N * W), and a token only needs the W - 1 keys before it plus the first k tokens, Sec. 3.2.1, so a stretch can
+ * be processed from local data once a halo of earlier keys and the sink rows have been brought in).
+ *   k_local, v_local [Tk, Hkv, D] packed by cu_k: for sequence b the keys at positions key_pos0[b] ..
+ *       key_pos0[b] + len_k - 1 (halo followed by the owned stretch);
+ *   q [Tq, Hq, D] packed by cu_q: the queries of the LAST len_q of those positions;
+ *   sink_k, sink_v [B, sink_rows, Hkv, D]: the keys at positions 0 .. sink_rows - 1 of every sequence.
+ * A query at position i sees the positions the mask policy allows; each is taken from the local keys when
+ * p >= key_pos0[b], else from the sink rows when p < min(S, sink_rows); a visible position available from
+ * neither (halo too short) is an error (-2).  Keys are visited in increasing position, exactly as
+ * swaa_oracle_prefill visits them.  Rows chosen as in swaa_oracle_prefill_chunked.
+ */
+int swaa_oracle_prefill_cp(const float* q, const float* k_local, const float* v_local, const float* sink_k,
+                           const float* sink_v, const int32_t* cu_q, const int32_t* cu_k, const int64_t* key_pos0,
+                           int B, int64_t sink_rows, int Hq, int Hkv, int D, int64_t W, int64_t S, int is_full,
+                           double scale, int64_t n_rows, const int64_t* row_t, const int32_t* row_h, double* out,
+                           double* lse, int64_t* nvis) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || Hq % Hkv != 0 || sink_rows < 0) return -1;
+    if (!is_full && W < 1) return -1;
+    if (S < 0) return -1;
+    const int G = Hq / Hkv;
+    const int64_t Tq = B > 0 ? cu_q[B] : 0;
+    int64_t max_pos = 0;
+    for (int b = 0; b < B; ++b) {
+        int64_t lq = (int64_t)cu_q[b + 1] - cu_q[b], lk = (int64_t)cu_k[b + 1] - cu_k[b];
+        if (lq < 0 || lk < lq || key_pos0[b] < 0) return -1;
+        if (key_pos0[b] + lk > max_pos) max_pos = key_pos0[b] + lk;
+    }
+    if (row_t == NULL && n_rows != Tq * Hq) return -1;
+    int bad = 0;
+#pragma omp parallel
+    {
+        double* scores = (double*)malloc(sizeof(double) * (size_t)(max_pos > 0 ? max_pos : 1));
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            const int64_t t = row_t ? row_t[r] : r / Hq;
+            const int h = row_t ? row_h[r] : (int)(r % Hq);
+            if (t < 0 || t >= Tq || h < 0 || h >= Hq) {
+#pragma omp atomic write
+                bad = 1;
+                continue;
+            }
+            int b = 0;
+            while (!(cu_q[b] <= t && t < cu_q[b + 1])) ++b;
+            const int64_t lq = (int64_t)cu_q[b + 1] - cu_q[b], lk = (int64_t)cu_k[b + 1] - cu_k[b];
+            const int64_t p0 = key_pos0[b];
+            const int64_t i = p0 + (lk - lq) + (t - cu_q[b]);
+            const int hk = h / G;
+            const float* qi = q + (t * Hq + h) * (int64_t)D;
+            double m = -INFINITY;
+            int64_t cnt = 0;
+            int missing = 0;
+            for (int64_t p = 0; p <= i; ++p) {
+                if (!swaa_oracle_visible(i, p, W, S, is_full)) continue;
+                const float* kp;
+                if (p >= p0) kp = k_local + ((cu_k[b] + (p - p0)) * Hkv + hk) * (int64_t)D;
+                else if (p < S && p < sink_rows) kp = sink_k + (((int64_t)b * sink_rows + p) * Hkv + hk) * D;
+                else { missing = 1; break; }
+                double sdot = 0.0;
+                for (int d = 0; d < D; ++d) sdot += (double)qi[d] * (double)kp[d];
+                scores[p] = sdot * scale;
+                if (scores[p] > m) m = scores[p];
+                ++cnt;
+            }
+            if (missing) {
+#pragma omp atomic write
+                bad = 2;
+                continue;
+            }
+            double denom = 0.0;
+            for (int64_t p = 0; p <= i; ++p)
+                if (swaa_oracle_visible(i, p, W, S, is_full)) denom += exp(scores[p] - m);
+            double* orow = out + r * D;
+            for (int d = 0; d < D; ++d) orow[d] = 0.0;
+            for (int64_t p = 0; p <= i; ++p) {
+                if (!swaa_oracle_visible(i, p, W, S, is_full)) continue;
+                const double pr = exp(scores[p] - m) / denom;
+                const float* vp = p >= p0 ? v_local + ((cu_k[b] + (p - p0)) * Hkv + hk) * (int64_t)D
+                                          : sink_v + (((int64_t)b * sink_rows + p) * Hkv + hk) * D;
+                for (int d = 0; d < D; ++d) orow[d] += pr * (double)vp[d];
+            }
+            if (lse) lse[r] = m + log(denom);
+            if (nvis) nvis[r] = cnt;
+        }
+        free(scores);
+    }
+    return bad == 0 ? 0 : -bad;
 }
 
 /*
@@ -532,6 +711,37 @@ int swaa_oracle_layer_is_full(int layer, int fa_start, int fa_step, int fa_decod
             if (l == layer) in_list = 1;
     if (in_list) return 1;
     if (phase == 1 && fa_decode) return 1;
+    return 0;
+}
+
+/*
+ * The same with an explicit set of FA layers (App. "Results of LightTransfer": the FA layers are chosen per layer
+ * by a lazy ratio instead of at a fixed interval): fa_mask[layer] != 0 marks an FA layer.
+ */
+int swaa_oracle_layer_is_full_mask(int layer, const uint8_t* fa_mask, int fa_decode, int phase) {
+    if (fa_mask[layer]) return 1;
+    if (phase == 1 && fa_decode) return 1;
+    return 0;
+}
+
+/*
+ * Layer selection by lazy ratio (App. "Results of LightTransfer"): the n_lazy layers with the HIGHEST ratio are the
+ * "lazy" ones (those that could take SWA), the rest "non-lazy".  fa_on_lazy == 0 gives full attention to the
+ * non-lazy layers (the method as proposed), != 0 to the lazy ones (the variant the paper also evaluates).  Equal
+ * ratios: the layer with the lower index counts as the lazier.  Plain selection: n_lazy passes, each taking the
+ * largest remaining ratio.  fa_mask_out [n_layers].
+ */
+int swaa_oracle_select_fa_layers(const double* ratio, int n_layers, int n_lazy, int fa_on_lazy, uint8_t* fa_mask_out) {
+    if (n_layers < 0 || n_lazy < 0 || n_lazy > n_layers) return -1;
+    uint8_t* lazy = (uint8_t*)calloc((size_t)(n_layers > 0 ? n_layers : 1), 1);
+    for (int pass = 0; pass < n_lazy; ++pass) {
+        int best = -1;
+        for (int l = 0; l < n_layers; ++l)
+            if (!lazy[l] && (best < 0 || ratio[l] > ratio[best])) best = l;
+        lazy[best] = 1;
+    }
+    for (int l = 0; l < n_layers; ++l) fa_mask_out[l] = (uint8_t)(fa_on_lazy ? lazy[l] : !lazy[l]);
+    free(lazy);
     return 0;
 }
 

@@ -45,8 +45,8 @@ def _load():
         lib.swaa_oracle_prefill.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl, i64,
                                             vp, vp, vp, vp, vp, vp]
         lib.swaa_oracle_prefill.restype = ctypes.c_int
-        lib.swaa_oracle_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, dbl,
-                                                    i64, vp, vp, vp, vp, vp, vp]
+        lib.swaa_oracle_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int, vp,
+                                                    dbl, i64, vp, vp, vp, vp, vp, vp]
         lib.swaa_oracle_prefill_chunked.restype = ctypes.c_int
         lib.swaa_oracle_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, ctypes.c_int,
                                                      dbl, vp, vp, vp]
@@ -59,6 +59,18 @@ def _load():
         lib.swaa_oracle_decode.restype = ctypes.c_int
         lib.swaa_oracle_layer_is_full.argtypes = [ctypes.c_int] * 5
         lib.swaa_oracle_layer_is_full.restype = ctypes.c_int
+        lib.swaa_oracle_layer_is_full_mask.argtypes = [ctypes.c_int, vp, ctypes.c_int, ctypes.c_int]
+        lib.swaa_oracle_layer_is_full_mask.restype = ctypes.c_int
+        lib.swaa_oracle_select_fa_layers.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
+        lib.swaa_oracle_select_fa_layers.restype = ctypes.c_int
+        lib.swaa_oracle_decode_partial.argtypes = [vp, vp, vp, vp, i32, i64, i64, i32, i32, i32, i64, i64, ctypes.c_int,
+                                                   dbl, vp, vp]
+        lib.swaa_oracle_decode_partial.restype = ctypes.c_int
+        lib.swaa_oracle_decode_combine.argtypes = [vp, ctypes.c_int, i64, ctypes.c_int, vp]
+        lib.swaa_oracle_decode_combine.restype = ctypes.c_int
+        lib.swaa_oracle_prefill_cp.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i64, i64,
+                                               ctypes.c_int, dbl, i64, vp, vp, vp, vp, vp]
+        lib.swaa_oracle_prefill_cp.restype = ctypes.c_int
         lib.swaa_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -127,11 +139,12 @@ def prefill(q, k, v, cu_seqlens, window: int, n_sink: int, is_full: bool, scale:
 
 
 def prefill_chunked(q, k, v, cu_seqlens_q, cu_seqlens_k, window: int, n_sink: int, is_full: bool,
-                    scale: float | None = None, rows=None):
+                    scale: float | None = None, rows=None, is_full_seq=None):
     """Chunked prefill: queries are the last len_q tokens of each sequence's len_k-token context.
 
     q [Tq,Hq,D] packed by cu_seqlens_q; k, v [Tk,Hkv,D] packed by cu_seqlens_k.  rows as in prefill()
-    (row_t indexes packed query tokens).  Returns a dict with out, lse, psum, nvis.
+    (row_t indexes packed query tokens).  is_full_seq (optional, [B]): a mask policy per sequence, replacing
+    is_full.  Returns a dict with out, lse, psum, nvis.
     """
     q, k, v = _f32(q), _f32(k), _f32(v)
     Tq, Hq, D = q.shape
@@ -154,8 +167,10 @@ def prefill_chunked(q, k, v, cu_seqlens_q, cu_seqlens_k, window: int, n_sink: in
     lse = np.empty(n_rows, dtype=np.float64)
     psum = np.empty(n_rows, dtype=np.float64)
     nvis = np.empty(n_rows, dtype=np.int64)
+    fs = None if is_full_seq is None else np.ascontiguousarray(np.asarray(is_full_seq, dtype=np.uint8))
+    assert fs is None or fs.shape == (B,)
     rc = _load().swaa_oracle_prefill_chunked(_ptr(q), _ptr(k), _ptr(v), _ptr(cq), _ptr(ck), B, Hq, Hkv, D, int(window),
-                                             int(n_sink), int(bool(is_full)), float(scale), n_rows, _ptr(rt), _ptr(rh),
+                                             int(n_sink), int(bool(is_full)), _ptr(fs), float(scale), n_rows, _ptr(rt), _ptr(rh),
                                              _ptr(out), _ptr(lse), _ptr(psum), _ptr(nvis))
     if rc != 0:
         raise ValueError("swaa_oracle_prefill_chunked: inconsistent arguments")
@@ -185,6 +200,94 @@ def decode(q, kcache, vcache, seqlens, window: int, n_sink: int, is_full: bool, 
     if rc != 0:
         raise ValueError("swaa_oracle_decode: inconsistent arguments")
     return {"out": out, "lse": lse, "psum": psum, "nvis": nvis}
+
+
+def decode_partial(q, kshard, vshard, seqlens, pos0: int, window: int, n_sink: int, is_full: bool,
+                   scale: float | None = None):
+    """Partial decode result of one shard of a cache cut along the context.  kshard, vshard [B,Lshard,Hkv,D] hold
+    positions pos0 .. pos0+Lshard-1 of every sequence; seqlens are the total lengths.  Returns part [B,Hq,D+2]
+    float64 = (max score, sum of exp, unnormalised output) and nvis [B,Hq]."""
+    q, kshard, vshard = _f32(q), _f32(kshard), _f32(vshard)
+    B, Hq, D = q.shape
+    _, Lshard, Hkv, _ = kshard.shape
+    assert kshard.shape == (B, Lshard, Hkv, D) and vshard.shape == kshard.shape
+    sl = np.ascontiguousarray(np.asarray(seqlens, dtype=np.int32))
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    part = np.empty((B, Hq, D + 2), dtype=np.float64)
+    nvis = np.empty((B, Hq), dtype=np.int64)
+    rc = _load().swaa_oracle_decode_partial(_ptr(q), _ptr(kshard), _ptr(vshard), _ptr(sl), B, Lshard, int(pos0), Hq, Hkv,
+                                            D, int(window), int(n_sink), int(bool(is_full)), float(scale), _ptr(part),
+                                            _ptr(nvis))
+    if rc != 0:
+        raise ValueError("swaa_oracle_decode_partial: inconsistent arguments")
+    return {"part": part, "nvis": nvis}
+
+
+def decode_combine(parts):
+    """Log-sum-exp combine of partial decode results.  parts [P,B,Hq,D+2] float64 -> out [B,Hq,D] float64."""
+    parts = np.ascontiguousarray(np.asarray(parts, dtype=np.float64))
+    P, B, Hq, D2 = parts.shape
+    out = np.empty((B, Hq, D2 - 2), dtype=np.float64)
+    rc = _load().swaa_oracle_decode_combine(_ptr(parts), P, B * Hq, D2 - 2, _ptr(out))
+    if rc != 0:
+        raise ValueError("swaa_oracle_decode_combine: inconsistent arguments")
+    return out
+
+
+def prefill_cp(q, k_local, v_local, sink_k, sink_v, cu_seqlens_q, cu_seqlens_k, key_pos0, window: int, n_sink: int,
+               is_full: bool, scale: float | None = None, rows=None):
+    """Context-parallel prefill of one participant (see swaa_oracle.c): local keys of sequence b start at position
+    key_pos0[b]; the queries are the last len_q local positions; sink_k, sink_v [B,sink_rows,Hkv,D] hold positions
+    0..sink_rows-1.  Raises ValueError when a visible key is available from neither.  Returns out, lse, nvis."""
+    q, k_local, v_local, sink_k, sink_v = _f32(q), _f32(k_local), _f32(v_local), _f32(sink_k), _f32(sink_v)
+    Tq, Hq, D = q.shape
+    Tk, Hkv, _ = k_local.shape
+    cq = np.ascontiguousarray(np.asarray(cu_seqlens_q, dtype=np.int32))
+    ck = np.ascontiguousarray(np.asarray(cu_seqlens_k, dtype=np.int32))
+    p0 = np.ascontiguousarray(np.asarray(key_pos0, dtype=np.int64))
+    B = cq.shape[0] - 1
+    assert ck.shape[0] == B + 1 and p0.shape == (B,) and cq[-1] == Tq and ck[-1] == Tk
+    sink_rows = sink_k.shape[1]
+    assert sink_k.shape == (B, sink_rows, Hkv, D) and sink_v.shape == sink_k.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    if rows is None:
+        n_rows, rt, rh = Tq * Hq, None, None
+    else:
+        rt = np.ascontiguousarray(np.asarray(rows[0], dtype=np.int64))
+        rh = np.ascontiguousarray(np.asarray(rows[1], dtype=np.int32))
+        n_rows = rt.shape[0]
+    out = np.empty((n_rows, D), dtype=np.float64)
+    lse = np.empty(n_rows, dtype=np.float64)
+    nvis = np.empty(n_rows, dtype=np.int64)
+    rc = _load().swaa_oracle_prefill_cp(_ptr(q), _ptr(k_local), _ptr(v_local), _ptr(sink_k), _ptr(sink_v), _ptr(cq),
+                                        _ptr(ck), _ptr(p0), B, sink_rows, Hq, Hkv, D, int(window), int(n_sink),
+                                        int(bool(is_full)), float(scale), n_rows, _ptr(rt), _ptr(rh), _ptr(out),
+                                        _ptr(lse), _ptr(nvis))
+    if rc == -2:
+        raise ValueError("swaa_oracle_prefill_cp: a visible key is in neither the local keys nor the sink rows")
+    if rc != 0:
+        raise ValueError("swaa_oracle_prefill_cp: inconsistent arguments")
+    if rows is None:
+        return {"out": out.reshape(Tq, Hq, D), "lse": lse.reshape(Tq, Hq), "nvis": nvis.reshape(Tq, Hq)}
+    return {"out": out, "lse": lse, "nvis": nvis}
+
+
+def layer_is_full_mask(layer: int, fa_mask, fa_decode: bool, phase: int) -> bool:
+    m = np.ascontiguousarray(np.asarray(fa_mask, dtype=np.uint8))
+    assert 0 <= layer < m.shape[0]
+    return bool(_load().swaa_oracle_layer_is_full_mask(int(layer), _ptr(m), int(bool(fa_decode)), int(phase)))
+
+
+def select_fa_layers(ratio, n_lazy: int, fa_on_lazy: bool):
+    """FA-layer set from per-layer lazy ratios (see swaa_oracle.c).  Returns a uint8 array [n_layers]."""
+    r = np.ascontiguousarray(np.asarray(ratio, dtype=np.float64))
+    out = np.zeros(r.shape[0], dtype=np.uint8)
+    rc = _load().swaa_oracle_select_fa_layers(_ptr(r), r.shape[0], int(n_lazy), int(bool(fa_on_lazy)), _ptr(out))
+    if rc != 0:
+        raise ValueError("swaa_oracle_select_fa_layers: inconsistent arguments")
+    return out
 
 
 def decode_paged(q, kpages, vpages, block_table, seqlens, window: int, n_sink: int, is_full: bool,
