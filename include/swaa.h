@@ -232,7 +232,10 @@ int swaa_decode_static(const void* q, const void* kcache, const void* vcache, vo
  * Layer schedule (host only).  Sec. 3.1.2: a fixed-interval subset of layers keeps full attention
  * (Table 1 "FA layers": [1,3,5,...], [0,2,4,...], [1,5,9,...], [1,9,17,...], [3,7,11,...]); Sec. 3.1.1:
  * with FA decode every layer is full while decoding.  Layers are 0-based.
- *   is_full(layer, phase) = (layer in {fa_start, fa_start+fa_step, ...}) or (phase == decode and fa_decode)
+ *   is_full(layer, phase) = (layer in FA set) or (phase == decode and fa_decode)
+ * The FA set is {fa_start, fa_start+fa_step, ...}, or, when fa_mask is not NULL, the layers l with fa_mask[l] != 0
+ * (a set chosen layer by layer, e.g. by lazy ratio as in App. "Results of LightTransfer"; fa_start and fa_step are
+ * then ignored).
  */
 typedef struct {
     int n_layers;
@@ -241,6 +244,7 @@ typedef struct {
     int fa_start;  /* first FA layer */
     int fa_step;   /* distance between FA layers; 0 = no FA layers */
     int fa_decode; /* non-zero: full attention in the decode phase on every layer */
+    const uint8_t* fa_mask; /* NULL, or host array [n_layers]: explicit FA set (owned by the caller) */
 } swaa_policy;
 
 #define SWAA_PHASE_PREFILL 0
@@ -250,6 +254,20 @@ typedef struct {
 int swaa_schedule_is_full(const swaa_policy* policy, int layer, int phase);
 /* Fills is_full_out[0 .. n_layers) (host memory) with 0/1.  Returns SWAA_OK or SWAA_ERR_INVALID_ARG. */
 int swaa_schedule_fill(const swaa_policy* policy, int phase, uint8_t* is_full_out);
+/*
+ * FA set from lazy ratios (host only; App. "Results of LightTransfer": layers with a higher lazy ratio are the
+ * candidates for SWA, the others keep full attention; the paper also evaluates the opposite assignment).
+ *   ratio       host, float32 [n_layers, n_heads]: per layer the output of swaa_lazy_ratio; a layer's ratio is the
+ *               mean over its heads.
+ *   n_lazy      how many layers count as lazy: those with the highest ratio (equal ratios: lower index first);
+ *               the paper takes half of the layers.
+ *   fa_on_lazy  0: the non-lazy layers get full attention (the method as proposed); != 0: the lazy ones do.
+ *   fa_mask_out host, uint8 [n_layers]: 1 for FA layers; usable as swaa_policy.fa_mask.
+ * Returns SWAA_OK or SWAA_ERR_INVALID_ARG (null pointer, n_layers < 0, n_heads < 1, n_lazy outside [0, n_layers],
+ * a ratio that is not finite).
+ */
+int swaa_schedule_select_fa_layers(const float* ratio, int n_layers, int n_heads, int n_lazy, int fa_on_lazy,
+                                   uint8_t* fa_mask_out);
 
 /*
  * Key-tile enumeration of the prefill kernel, exposed for host-side verification (App. A: only

@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     load_library,
     schedule_fill,
     schedule_is_full,
+    schedule_select_fa_layers,
     status_str,
     swaa_decode,
     swaa_decode_paged,

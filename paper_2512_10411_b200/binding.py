@@ -29,7 +29,8 @@ class SwaaError(RuntimeError):
 
 
 class _Policy(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int) for n in ("n_layers", "window", "n_sink", "fa_start", "fa_step", "fa_decode")]
+    _fields_ = [(n, ctypes.c_int) for n in ("n_layers", "window", "n_sink", "fa_start", "fa_step", "fa_decode")] + \
+               [("fa_mask", ctypes.POINTER(ctypes.c_uint8))]
 
 
 @dataclass
@@ -41,9 +42,18 @@ class SwaaPolicy:
     fa_start: int = 0
     fa_step: int = 0
     fa_decode: bool = False
+    fa_mask: list | None = None  # explicit FA set: one 0/1 entry per layer (replaces fa_start / fa_step)
 
     def _c(self) -> _Policy:
-        return _Policy(self.n_layers, self.window, self.n_sink, self.fa_start, self.fa_step, int(bool(self.fa_decode)))
+        mask = None
+        if self.fa_mask is not None:
+            if len(self.fa_mask) != self.n_layers:
+                raise ValueError("SwaaPolicy.fa_mask must have n_layers entries")
+            mask = (ctypes.c_uint8 * max(self.n_layers, 1))(*[int(bool(x)) for x in self.fa_mask])
+        c = _Policy(self.n_layers, self.window, self.n_sink, self.fa_start, self.fa_step, int(bool(self.fa_decode)),
+                    ctypes.cast(mask, ctypes.POINTER(ctypes.c_uint8)) if mask is not None else None)
+        c._keepalive = mask  # the C struct only borrows the array
+        return c
 
 
 def lib_path() -> str:
@@ -88,6 +98,9 @@ def load_library():
     lib.swaa_schedule_is_full.restype = ci
     lib.swaa_schedule_fill.argtypes = [ctypes.POINTER(_Policy), ci, ctypes.POINTER(ctypes.c_uint8)]
     lib.swaa_schedule_fill.restype = ci
+    lib.swaa_schedule_select_fa_layers.argtypes = [ctypes.POINTER(ctypes.c_float), ci, ci, ci, ci,
+                                                   ctypes.POINTER(ctypes.c_uint8)]
+    lib.swaa_schedule_select_fa_layers.restype = ci
     lib.swaa_prefill_tile_range.argtypes = [ci] * 7 + [ctypes.POINTER(ci)] * 3
     lib.swaa_prefill_tile_range.restype = ci
     lib.swaa_prefill_tile_needs_mask.argtypes = [ci] * 8
@@ -352,6 +365,22 @@ def schedule_fill(policy: SwaaPolicy, phase: int) -> list:
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_schedule_fill")
     return [bool(buf[i]) for i in range(policy.n_layers)]
+
+
+def schedule_select_fa_layers(ratio, n_lazy: int, fa_on_lazy: bool) -> list:
+    """Forwards to C swaa_schedule_select_fa_layers.  ratio: [n_layers][n_heads] numbers on the host (per layer the
+    output of swaa_lazy_ratio).  Returns the FA mask as a list of 0/1, usable as SwaaPolicy.fa_mask."""
+    rows = [list(map(float, r)) for r in ratio]
+    n_layers = len(rows)
+    n_heads = len(rows[0]) if n_layers else 1
+    if any(len(r) != n_heads for r in rows):
+        raise ValueError("schedule_select_fa_layers: ragged ratio table")
+    flat = (ctypes.c_float * max(n_layers * n_heads, 1))(*[x for r in rows for x in r])
+    out = (ctypes.c_uint8 * max(n_layers, 1))()
+    rc = load_library().swaa_schedule_select_fa_layers(flat, n_layers, n_heads, int(n_lazy), int(bool(fa_on_lazy)), out)
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_schedule_select_fa_layers")
+    return [int(out[i]) for i in range(n_layers)]
 
 
 def prefill_tile_range(L, m, BM, BN, window, n_sink, is_full):

@@ -4,8 +4,11 @@
 #include <math.h>
 #include <stdint.h>
 
+#include <algorithm>
+#include <cmath>
 #include <mutex>
 #include <random>
+#include <vector>
 
 #include "swaa.h"
 #include "swaa_internal.cuh"
@@ -673,6 +676,7 @@ extern "C" int swaa_schedule_is_full(const swaa_policy* policy, int layer, int p
     if (phase != SWAA_PHASE_PREFILL && phase != SWAA_PHASE_DECODE) return SWAA_ERR_INVALID_ARG;
     if (policy->fa_start < 0 || policy->fa_step < 0) return SWAA_ERR_INVALID_ARG;
     if (phase == SWAA_PHASE_DECODE && policy->fa_decode) return 1;
+    if (policy->fa_mask != nullptr) return policy->fa_mask[layer] != 0 ? 1 : 0;
     if (policy->fa_step > 0 && layer >= policy->fa_start && (layer - policy->fa_start) % policy->fa_step == 0) return 1;
     return 0;
 }
@@ -683,6 +687,28 @@ extern "C" int swaa_schedule_fill(const swaa_policy* policy, int phase, uint8_t*
         const int r = swaa_schedule_is_full(policy, l, phase);
         if (r < 0) return r;
         is_full_out[l] = (uint8_t)r;
+    }
+    return SWAA_OK;
+}
+
+extern "C" int swaa_schedule_select_fa_layers(const float* ratio, int n_layers, int n_heads, int n_lazy, int fa_on_lazy,
+                                              uint8_t* fa_mask_out) {
+    if (!ratio || !fa_mask_out || n_layers < 0 || n_heads < 1 || n_lazy < 0 || n_lazy > n_layers)
+        return SWAA_ERR_INVALID_ARG;
+    std::vector<double> mean((size_t)n_layers);
+    std::vector<int> order((size_t)n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+        double acc = 0.0;
+        for (int h = 0; h < n_heads; ++h) acc += (double)ratio[(size_t)l * n_heads + h];
+        if (!std::isfinite(acc)) return SWAA_ERR_INVALID_ARG;
+        mean[(size_t)l] = acc / n_heads;
+        order[(size_t)l] = l;
+    }
+    // laziest first; the stable sort keeps the lower index ahead among equal ratios
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return mean[(size_t)a] > mean[(size_t)b]; });
+    for (int r = 0; r < n_layers; ++r) {
+        const bool lazy = r < n_lazy;
+        fa_mask_out[order[(size_t)r]] = (uint8_t)((fa_on_lazy != 0) == lazy ? 1 : 0);
     }
     return SWAA_OK;
 }

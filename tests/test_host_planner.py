@@ -99,6 +99,42 @@ def test_schedule_matches_paper_patterns():
                 assert [swaa.schedule_is_full(pol, l, phase) for l in range(36)] == want
 
 
+def test_schedule_with_an_explicit_fa_layer_set():
+    """A non-periodic FA set (what a selection by lazy ratio produces) against the oracle, in both phases."""
+    rng = np.random.default_rng(8)
+    for n_layers in (1, 7, 36):
+        mask = rng.integers(0, 2, n_layers).tolist()
+        for fa_decode in (False, True):
+            pol = swaa.SwaaPolicy(n_layers, 2048, 100, 3, 4, fa_decode, fa_mask=mask)  # start / step are ignored
+            for phase in (0, 1):
+                want = [oracle.layer_is_full_mask(l, mask, fa_decode, phase) for l in range(n_layers)]
+                assert swaa.schedule_fill(pol, phase) == want
+                assert [swaa.schedule_is_full(pol, l, phase) for l in range(n_layers)] == want
+    with pytest.raises(ValueError):
+        swaa.schedule_fill(swaa.SwaaPolicy(4, 8, 0, 0, 0, False, fa_mask=[1, 0]), 0)
+
+
+def test_fa_layers_selected_by_lazy_ratio():
+    """Per-head ratios as swaa_lazy_ratio returns them -> per-layer mean -> the half with the higher ratio is "lazy";
+    FA on the non-lazy half (the method as proposed) or on the lazy half (the variant of the paper's LightTransfer
+    table), against the oracle's plain selection; ties, sizes and argument errors."""
+    rng = np.random.default_rng(9)
+    for n_layers, n_heads, n_lazy in ((36, 32, 18), (36, 8, 27), (5, 1, 0), (5, 3, 5), (1, 2, 1)):
+        table = rng.random((n_layers, n_heads)).astype(np.float32)
+        per_layer = table.astype(np.float64).mean(axis=1)
+        for fa_on_lazy in (False, True):
+            got = swaa.schedule_select_fa_layers(table, n_lazy, fa_on_lazy)
+            assert got == oracle.select_fa_layers(per_layer, n_lazy, fa_on_lazy).tolist()
+            assert sum(got) == (n_lazy if fa_on_lazy else n_layers - n_lazy)
+            pol = swaa.SwaaPolicy(n_layers, 2048, 100, fa_decode=True, fa_mask=got)
+            assert swaa.schedule_fill(pol, 0) == [bool(x) for x in got] and all(swaa.schedule_fill(pol, 1))
+    assert swaa.schedule_select_fa_layers([[0.5], [0.5], [0.5], [0.5]], 2, True) == [1, 1, 0, 0]
+    with pytest.raises(swaa.SwaaError):
+        swaa.schedule_select_fa_layers([[0.1], [0.2]], 3, True)
+    with pytest.raises(swaa.SwaaError):
+        swaa.schedule_select_fa_layers([[0.1], [float("nan")]], 1, True)
+
+
 def test_schedule_argument_errors():
     pol = swaa.SwaaPolicy(4, 8, 0, 1, 2, False)
     for layer, phase in ((-1, 0), (4, 0), (0, 2)):
