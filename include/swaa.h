@@ -135,6 +135,50 @@ int swaa_prefill_paged(const void* q, const void* kpages, const void* vpages, vo
                        int is_full, float scale, float* lse, void* stream);
 
 /*
+ * Mixed batch: swaa_prefill_chunked / swaa_prefill_paged with a mask policy PER SEQUENCE, so that one launch serves
+ * sequences in different phases (Fig. 1a: prompt tokens under the SWA mask next to generated tokens under full
+ * attention; App. "Inference Efficiency": a serving engine batches prefill chunks and decode tokens together).
+ *   is_full_seq   device, uint8 [B]; sequence b runs full causal attention iff is_full_seq[b] != 0, else the
+ *                 window + n_sink mask.  window >= 1 is required.
+ * Everything else as for swaa_prefill_chunked / swaa_prefill_paged.
+ */
+int swaa_prefill_chunked_mixed(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens_q,
+                               const int32_t* cu_seqlens_k, const uint8_t* is_full_seq, int B, int Tq, int Tk,
+                               int max_seqlen_q, int max_seqlen_k, int Hq, int Hkv, int D, int window, int n_sink,
+                               float scale, float* lse, void* stream);
+int swaa_prefill_paged_mixed(const void* q, const void* kpages, const void* vpages, void* out,
+                             const int32_t* cu_seqlens_q, const int32_t* seqlens_k, const int32_t* block_table,
+                             const uint8_t* is_full_seq, int B, int Tq, int max_seqlen_q, int max_blocks, int num_pages,
+                             int page_size, int Hq, int Hkv, int D, int window, int n_sink, float scale, float* lse,
+                             void* stream);
+
+/*
+ * Context-parallel SWA prefill: the compute step of one participant that owns a contiguous stretch of every
+ * sequence (App. A: SWA prefill costs O(N * W) because a token only looks at the window before it; Sec. 3.2.1: and
+ * at the first k tokens).  Before the call the participant has, in its own memory,
+ *   k_local, v_local  device, [Tk, Hkv, D] bf16 packed by cu_seqlens_k: for sequence b the keys at positions
+ *                     key_pos0[b] .. key_pos0[b] + len_k - 1, i.e. a halo of earlier keys followed by its stretch;
+ *   q, out            device, [Tq, Hq, D] bf16 packed by cu_seqlens_q: the LAST len_q of those positions (its stretch);
+ *   sink_k, sink_v    device, [B, sink_rows, Hkv, D] bf16: the keys at positions 0 .. sink_rows-1 of every sequence
+ *                     (finite values in every row); may be NULL with sink_rows == 0 when n_sink == 0 or every
+ *                     key_pos0 is 0;
+ *   key_pos0          device, int32 [B].
+ * How halo and sink rows get there (a neighbour copy and a broadcast) is the caller's business; the kernel reads
+ * local memory only.  A query at position i sees positions j <= i with j > i - window or j < n_sink: positions
+ * >= key_pos0[b] are taken from the local keys, sink positions below it from the sink rows.  The halo must hold
+ * the window of the stretch's first query: key_pos0[b] == 0 or len_k - len_q >= window - 1, and n_sink <= sink_rows
+ * when key_pos0[b] > 0; a sequence that violates this is reported as SWAA_ERR_BAD_SEQLENS through the status word
+ * and its rows are not written.  With every key_pos0 == 0 this is swaa_prefill_chunked with the SWA mask.
+ * Layers with full attention need all earlier keys, i.e. an all-gather of K and V and then swaa_prefill_chunked.
+ * Other arguments as for swaa_prefill_chunked.
+ */
+int swaa_prefill_context_parallel(const void* q, const void* k_local, const void* v_local, const void* sink_k,
+                                  const void* sink_v, void* out, const int32_t* cu_seqlens_q,
+                                  const int32_t* cu_seqlens_k, const int32_t* key_pos0, int B, int Tq, int Tk,
+                                  int max_seqlen_q, int max_seqlen_k, int sink_rows, int Hq, int Hkv, int D, int window,
+                                  int n_sink, float scale, float* lse, void* stream);
+
+/*
  * Lazy ratio of a layer (App. "Results of LightTransfer": layer selection by how much of the attention of the
  * tokens at the end of a sequence goes to recent tokens rather than to the rest of the context; the paper
  * uses the last 64 tokens and a recent window of 1024).  For the queries given (the last len_q tokens of each

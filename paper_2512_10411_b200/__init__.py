@@ -30,6 +30,7 @@ from .binding import (  # noqa: F401
     swaa_prefill_backward,
     prefill_backward_workspace_size,
     swaa_prefill_chunked,
+    swaa_prefill_context_parallel,
     swaa_prefill_paged,
     last_device_status,
     trimmed_cache_len,

@@ -74,6 +74,14 @@ def load_library():
     lib.swaa_prefill.restype = ci
     lib.swaa_prefill_chunked.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     lib.swaa_prefill_chunked.restype = ci
+    lib.swaa_prefill_chunked_mixed.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp]
+    lib.swaa_prefill_chunked_mixed.restype = ci
+    lib.swaa_prefill_paged_mixed.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf,
+                                             vp, vp]
+    lib.swaa_prefill_paged_mixed.restype = ci
+    lib.swaa_prefill_context_parallel.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci,
+                                                  ci, ci, cf, vp, vp]
+    lib.swaa_prefill_context_parallel.restype = ci
     lib.swaa_prefill_backward_workspace_size.argtypes = [ci, ci, ci, ci, ci, ci]
     lib.swaa_prefill_backward_workspace_size.restype = ctypes.c_size_t
     lib.swaa_prefill_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -163,8 +171,9 @@ def swaa_prefill(q, k, v, out, cu_seqlens, max_seqlen: int, window: int, n_sink:
 
 
 def swaa_prefill_chunked(q, k, v, out, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, window: int,
-                         n_sink: int, is_full: bool, scale: float = 0.0, lse=None, stream=None) -> None:
-    """Forwards to C swaa_prefill_chunked.  q, out [Tq,Hq,D]; k, v [Tk,Hkv,D] bf16; cu_seqlens_* int32 [B+1];
+                         n_sink: int, is_full: bool, scale: float = 0.0, lse=None, stream=None, is_full_seq=None) -> None:
+    """Forwards to C swaa_prefill_chunked, or, when is_full_seq (uint8 [B], a mask policy per sequence) is given, to
+    C swaa_prefill_chunked_mixed.  q, out [Tq,Hq,D]; k, v [Tk,Hkv,D] bf16; cu_seqlens_* int32 [B+1];
     lse f32 [Hq,Tq].  The queries of each sequence are the last len_q tokens of its len_k-token context."""
     lib = load_library()
     Tq, Hq, D = q.shape
@@ -177,6 +186,18 @@ def swaa_prefill_chunked(q, k, v, out, cu_seqlens_q, cu_seqlens_k, max_seqlen_q:
     if lse is not None and tuple(lse.shape) != (Hq, Tq):
         raise ValueError("swaa_prefill_chunked: lse must be [Hq, Tq]")
     bf = torch.bfloat16
+    if is_full_seq is not None:
+        if is_full_seq.numel() != B:
+            raise ValueError("swaa_prefill_chunked: is_full_seq must have one entry per sequence")
+        rc = lib.swaa_prefill_chunked_mixed(_dev_ptr(q, bf, "q"), _dev_ptr(k, bf, "k"), _dev_ptr(v, bf, "v"),
+                                            _dev_ptr(out, bf, "out"), _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
+                                            _dev_ptr(cu_seqlens_k, torch.int32, "cu_seqlens_k"),
+                                            _dev_ptr(is_full_seq, torch.uint8, "is_full_seq"), B, Tq, Tk,
+                                            int(max_seqlen_q), int(max_seqlen_k), Hq, Hkv, D, int(window), int(n_sink),
+                                            float(scale), _dev_ptr(lse, torch.float32, "lse"), _stream_ptr(stream))
+        if rc != SWAA_OK:
+            raise SwaaError(rc, "swaa_prefill_chunked_mixed")
+        return
     rc = lib.swaa_prefill_chunked(_dev_ptr(q, bf, "q"), _dev_ptr(k, bf, "k"), _dev_ptr(v, bf, "v"),
                                   _dev_ptr(out, bf, "out"), _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
                                   _dev_ptr(cu_seqlens_k, torch.int32, "cu_seqlens_k"), B, Tq, Tk, int(max_seqlen_q),
@@ -215,8 +236,8 @@ def swaa_prefill_backward(q, k, v, out, dout, lse, cu_seqlens, max_seqlen: int, 
 
 
 def swaa_prefill_paged(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, block_table, max_seqlen_q: int, window: int,
-                       n_sink: int, is_full: bool, scale: float = 0.0, lse=None, stream=None) -> None:
-    """Forwards to C swaa_prefill_paged.  q, out [Tq,Hq,D]; kpages, vpages [num_pages,page_size,Hkv,D] bf16;
+                       n_sink: int, is_full: bool, scale: float = 0.0, lse=None, stream=None, is_full_seq=None) -> None:
+    """Forwards to C swaa_prefill_paged (to C swaa_prefill_paged_mixed when is_full_seq, uint8 [B], is given).  q, out [Tq,Hq,D]; kpages, vpages [num_pages,page_size,Hkv,D] bf16;
     cu_seqlens_q int32 [B+1]; seqlens_k int32 [B]; block_table int32 [B,max_blocks]; lse f32 [Hq,Tq]."""
     lib = load_library()
     Tq, Hq, D = q.shape
@@ -229,6 +250,21 @@ def swaa_prefill_paged(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, block_ta
     if lse is not None and tuple(lse.shape) != (Hq, Tq):
         raise ValueError("swaa_prefill_paged: lse must be [Hq, Tq]")
     bf = torch.bfloat16
+    if is_full_seq is not None:
+        if is_full_seq.numel() != B:
+            raise ValueError("swaa_prefill_paged: is_full_seq must have one entry per sequence")
+        rc = lib.swaa_prefill_paged_mixed(_dev_ptr(q, bf, "q"), _dev_ptr(kpages, bf, "kpages"),
+                                          _dev_ptr(vpages, bf, "vpages"), _dev_ptr(out, bf, "out"),
+                                          _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
+                                          _dev_ptr(seqlens_k, torch.int32, "seqlens_k"),
+                                          _dev_ptr(block_table, torch.int32, "block_table"),
+                                          _dev_ptr(is_full_seq, torch.uint8, "is_full_seq"), B, Tq, int(max_seqlen_q),
+                                          block_table.shape[1], num_pages, page_size, Hq, Hkv, D, int(window),
+                                          int(n_sink), float(scale), _dev_ptr(lse, torch.float32, "lse"),
+                                          _stream_ptr(stream))
+        if rc != SWAA_OK:
+            raise SwaaError(rc, "swaa_prefill_paged_mixed")
+        return
     rc = lib.swaa_prefill_paged(_dev_ptr(q, bf, "q"), _dev_ptr(kpages, bf, "kpages"), _dev_ptr(vpages, bf, "vpages"),
                                 _dev_ptr(out, bf, "out"), _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
                                 _dev_ptr(seqlens_k, torch.int32, "seqlens_k"),
@@ -238,6 +274,39 @@ def swaa_prefill_paged(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, block_ta
                                 _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_prefill_paged")
+
+
+def swaa_prefill_context_parallel(q, k_local, v_local, sink_k, sink_v, out, cu_seqlens_q, cu_seqlens_k, key_pos0,
+                                  max_seqlen_q: int, max_seqlen_k: int, window: int, n_sink: int, scale: float = 0.0,
+                                  lse=None, stream=None) -> None:
+    """Forwards to C swaa_prefill_context_parallel.  q, out [Tq,Hq,D]; k_local, v_local [Tk,Hkv,D] bf16 (halo + own
+    stretch, starting at position key_pos0[b]); sink_k, sink_v [B,sink_rows,Hkv,D] bf16 or None; key_pos0 int32 [B]."""
+    lib = load_library()
+    Tq, Hq, D = q.shape
+    Tk, Hkv = k_local.shape[0], k_local.shape[1]
+    if tuple(k_local.shape) != (Tk, Hkv, D) or tuple(v_local.shape) != (Tk, Hkv, D) or tuple(out.shape) != (Tq, Hq, D):
+        raise ValueError("swaa_prefill_context_parallel: inconsistent tensor shapes")
+    B = cu_seqlens_q.numel() - 1
+    if cu_seqlens_k.numel() != B + 1 or key_pos0.numel() != B:
+        raise ValueError("swaa_prefill_context_parallel: cu_seqlens_k must be [B+1] and key_pos0 [B]")
+    sink_rows = 0
+    if sink_k is not None:
+        sink_rows = sink_k.shape[1]
+        if tuple(sink_k.shape) != (B, sink_rows, Hkv, D) or tuple(sink_v.shape) != tuple(sink_k.shape):
+            raise ValueError("swaa_prefill_context_parallel: sink_k, sink_v must be [B, sink_rows, Hkv, D]")
+    if lse is not None and tuple(lse.shape) != (Hq, Tq):
+        raise ValueError("swaa_prefill_context_parallel: lse must be [Hq, Tq]")
+    bf = torch.bfloat16
+    rc = lib.swaa_prefill_context_parallel(_dev_ptr(q, bf, "q"), _dev_ptr(k_local, bf, "k_local"),
+                                           _dev_ptr(v_local, bf, "v_local"), _dev_ptr(sink_k, bf, "sink_k"),
+                                           _dev_ptr(sink_v, bf, "sink_v"), _dev_ptr(out, bf, "out"),
+                                           _dev_ptr(cu_seqlens_q, torch.int32, "cu_seqlens_q"),
+                                           _dev_ptr(cu_seqlens_k, torch.int32, "cu_seqlens_k"),
+                                           _dev_ptr(key_pos0, torch.int32, "key_pos0"), B, Tq, Tk, int(max_seqlen_q),
+                                           int(max_seqlen_k), sink_rows, Hq, Hkv, D, int(window), int(n_sink),
+                                           float(scale), _dev_ptr(lse, torch.float32, "lse"), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_prefill_context_parallel")
 
 
 def swaa_lazy_ratio(q, k, v, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, recent: int, n_sink: int,

@@ -306,7 +306,8 @@ static int make_accum_map(CUtensorMap* map, const float* base, int T, int H, int
 
 template <int D, int kMode>
 static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                          const PrefillParams& p, int sm_count, cudaStream_t st) {
+                          const CUtensorMap& tsk, const CUtensorMap& tsv, const PrefillParams& p, int sm_count,
+                          cudaStream_t st) {
     using L = PrefillSmem<D>;
     if (cudaFuncSetAttribute(prefill_kernel<D, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              L::kDynamicBytes) != cudaSuccess)
@@ -314,7 +315,7 @@ static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CU
     // persistent blocks: one per SM (or fewer when there is less work), each walks its share of the items
     long long blocks = (long long)p.n_pairs * p.tiles_ub;
     if (blocks > sm_count) blocks = sm_count;
-    prefill_kernel<D, kMode><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, p);
+    prefill_kernel<D, kMode><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, tsk, tsv, p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
@@ -330,16 +331,32 @@ struct PagedKV {  // keys and values in pages (null block_table: packed layout)
     int max_blocks = 0, num_pages = 0, page_size = 0;
 };
 
+struct PrefillExtras {
+    const uint8_t* is_full_seq = nullptr;  // mask policy per sequence (chunked / paged)
+    // context-parallel prefill: local keys start at key_pos0[b]; sink rows in [B, sink_rows, Hkv, D] buffers
+    bool context_parallel = false;
+    const int32_t* key_pos0 = nullptr;
+    const void* sink_k = nullptr;
+    const void* sink_v = nullptr;
+    int sink_rows = 0;
+};
+
 static int prefill_impl(const void* q, const void* k, const void* v, void* out, const int32_t* cu_seqlens_q,
                         const int32_t* cu_seqlens_k, int B, int Tq, int Tk, int max_seqlen_q, int max_seqlen_k, int Hq,
                         int Hkv, int D, int window, int n_sink, int is_full, float scale, float* lse, void* stream,
-                        const PagedKV& paged = PagedKV()) {
+                        const PagedKV& paged = PagedKV(), const PrefillExtras& ex = PrefillExtras()) {
     if (B < 0 || Tq < 0 || Tk < 0 || max_seqlen_q < 0 || max_seqlen_k < 0 || Hq < 1 || Hkv < 1 || n_sink < 0)
         return SWAA_ERR_INVALID_ARG;
-    if (!is_full && window < 1) return SWAA_ERR_INVALID_ARG;
+    if ((!is_full || ex.is_full_seq != nullptr) && window < 1) return SWAA_ERR_INVALID_ARG;
     if (Hq % Hkv != 0 || (D != 64 && D != 128)) return SWAA_ERR_UNSUPPORTED;
     if (B == 0 || Tq == 0) return SWAA_OK;
     if (!q || !k || !v || !out || !cu_seqlens_q) return SWAA_ERR_INVALID_ARG;
+    if (ex.context_parallel) {
+        if (!ex.key_pos0 || ex.sink_rows < 0 || (reinterpret_cast<uintptr_t>(ex.key_pos0) & 3u) != 0)
+            return SWAA_ERR_INVALID_ARG;
+        if (ex.sink_rows > 0 && (!ex.sink_k || !ex.sink_v || !aligned16(ex.sink_k) || !aligned16(ex.sink_v)))
+            return SWAA_ERR_INVALID_ARG;
+    }
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(cu_seqlens_q) & 3u) != 0 || (reinterpret_cast<uintptr_t>(cu_seqlens_k) & 3u) != 0 ||
         (reinterpret_cast<uintptr_t>(lse) & 3u) != 0)
@@ -361,6 +378,11 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
         if ((rc = make_token_major_map(&tv, v, Tk, Hkv, D)) != SWAA_OK) return rc;
     }
     if ((rc = make_token_major_map(&to, out, Tq, Hq, D, 32)) != SWAA_OK) return rc;  // output rows, 32 at a time
+    CUtensorMap tsk = tk, tsv = tv;  // only the context-parallel instance reads these
+    if (ex.context_parallel && ex.sink_rows > 0) {  // (D, Hkv, sink_rows, B); rows past sink_rows read as zeros
+        if ((rc = make_cache_map(&tsk, ex.sink_k, B, ex.sink_rows, Hkv, D, kPrefillBN)) != SWAA_OK) return rc;
+        if ((rc = make_cache_map(&tsv, ex.sink_v, B, ex.sink_rows, Hkv, D, kPrefillBN)) != SWAA_OK) return rc;
+    }
 
     PrefillParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
@@ -389,21 +411,33 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
     if (p.tiles_ub == 0) return SWAA_OK;  // max_seqlen == 0: nothing can be valid
     // a window that covers the longest key sequence is full causal attention for every row; clamping keeps the
     // kernel's 32-bit column arithmetic (column - window) far from overflow
-    if (!is_full && max_seqlen_k >= 1 && window > max_seqlen_k) window = max_seqlen_k;
+    // (context-parallel: positions are offset by key_pos0, so the bound there is a constant far above any length)
+    if (ex.context_parallel) {
+        if (window > (1 << 30)) window = 1 << 30;
+    } else if (!is_full && max_seqlen_k >= 1 && window > max_seqlen_k) {
+        window = max_seqlen_k;
+    }
     p.window = window;
     p.n_sink = n_sink;
     p.is_full = is_full ? 1 : 0;
+    p.is_full_seq = ex.is_full_seq;
+    p.key_pos0 = ex.key_pos0;
+    // with no sink rows supplied only a participant whose keys start at position 0 can have sink keys
+    p.sink_rows = ex.sink_rows;
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)D);
     p.sl2 = p.scale * 1.4426950408889634f;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (ex.context_parallel)
+        return D == 128 ? launch_prefill<128, 3>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st)
+                        : launch_prefill<64, 3>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st);
     if (is_paged)
-        return D == 128 ? launch_prefill<128, 2>(tq, tk, tv, to, p, info.sm_count, st)
-                        : launch_prefill<64, 2>(tq, tk, tv, to, p, info.sm_count, st);
+        return D == 128 ? launch_prefill<128, 2>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st)
+                        : launch_prefill<64, 2>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st);
     if (cu_seqlens_k != nullptr)
-        return D == 128 ? launch_prefill<128, 1>(tq, tk, tv, to, p, info.sm_count, st)
-                        : launch_prefill<64, 1>(tq, tk, tv, to, p, info.sm_count, st);
-    return D == 128 ? launch_prefill<128, 0>(tq, tk, tv, to, p, info.sm_count, st)
-                    : launch_prefill<64, 0>(tq, tk, tv, to, p, info.sm_count, st);
+        return D == 128 ? launch_prefill<128, 1>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st)
+                        : launch_prefill<64, 1>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st);
+    return D == 128 ? launch_prefill<128, 0>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st)
+                    : launch_prefill<64, 0>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st);
 }
 
 }  // namespace swaa
@@ -439,6 +473,55 @@ extern "C" int swaa_prefill_paged(const void* q, const void* kpages, const void*
     pg.page_size = page_size;
     return prefill_impl(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, B, Tq, 0, max_seqlen_q, max_blocks * page_size, Hq,
                         Hkv, D, window, n_sink, is_full, scale, lse, stream, pg);
+}
+
+extern "C" int swaa_prefill_chunked_mixed(const void* q, const void* k, const void* v, void* out,
+                                          const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,
+                                          const uint8_t* is_full_seq, int B, int Tq, int Tk, int max_seqlen_q,
+                                          int max_seqlen_k, int Hq, int Hkv, int D, int window, int n_sink, float scale,
+                                          float* lse, void* stream) {
+    if (!cu_seqlens_k || !is_full_seq) return SWAA_ERR_INVALID_ARG;
+    PrefillExtras ex;
+    ex.is_full_seq = is_full_seq;
+    return prefill_impl(q, k, v, out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq, Hkv, D,
+                        window, n_sink, 0, scale, lse, stream, PagedKV(), ex);
+}
+
+extern "C" int swaa_prefill_paged_mixed(const void* q, const void* kpages, const void* vpages, void* out,
+                                        const int32_t* cu_seqlens_q, const int32_t* seqlens_k,
+                                        const int32_t* block_table, const uint8_t* is_full_seq, int B, int Tq,
+                                        int max_seqlen_q, int max_blocks, int num_pages, int page_size, int Hq, int Hkv,
+                                        int D, int window, int n_sink, float scale, float* lse, void* stream) {
+    if (!seqlens_k || !block_table || !is_full_seq) return SWAA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(block_table) & 3u) != 0) return SWAA_ERR_INVALID_ARG;
+    if (max_blocks < 1 || num_pages < 1 || page_size < 1) return SWAA_ERR_INVALID_ARG;
+    if (page_size % kPrefillBN != 0 || (long long)max_blocks * page_size > 2147483647LL) return SWAA_ERR_UNSUPPORTED;
+    PagedKV pg;
+    pg.block_table = block_table;
+    pg.max_blocks = max_blocks;
+    pg.num_pages = num_pages;
+    pg.page_size = page_size;
+    PrefillExtras ex;
+    ex.is_full_seq = is_full_seq;
+    return prefill_impl(q, kpages, vpages, out, cu_seqlens_q, seqlens_k, B, Tq, 0, max_seqlen_q, max_blocks * page_size, Hq,
+                        Hkv, D, window, n_sink, 0, scale, lse, stream, pg, ex);
+}
+
+extern "C" int swaa_prefill_context_parallel(const void* q, const void* k_local, const void* v_local,
+                                             const void* sink_k, const void* sink_v, void* out,
+                                             const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,
+                                             const int32_t* key_pos0, int B, int Tq, int Tk, int max_seqlen_q,
+                                             int max_seqlen_k, int sink_rows, int Hq, int Hkv, int D, int window,
+                                             int n_sink, float scale, float* lse, void* stream) {
+    if (!cu_seqlens_k || !key_pos0) return SWAA_ERR_INVALID_ARG;
+    PrefillExtras ex;
+    ex.context_parallel = true;
+    ex.key_pos0 = key_pos0;
+    ex.sink_k = sink_k;
+    ex.sink_v = sink_v;
+    ex.sink_rows = sink_rows;
+    return prefill_impl(q, k_local, v_local, out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq,
+                        Hkv, D, window, n_sink, 0, scale, lse, stream, PagedKV(), ex);
 }
 
 // -------------------------------------------------------------------------------------- backward

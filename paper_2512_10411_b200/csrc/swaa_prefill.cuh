@@ -52,6 +52,11 @@ struct PrefillParams {
     int n_pairs;            // Hkv * pairs_per_kv
     int tiles_ub;           // upper bound on the number of query tiles over all sequences
     int window, n_sink, is_full;
+    const uint8_t* is_full_seq;   // nullable (chunked / paged): mask policy per sequence, replaces is_full
+    // context-parallel prefill (kMode 3): the local keys of sequence b start at position key_pos0[b]; the keys at
+    // positions 0 .. sink_rows-1 of every sequence come from a separate buffer [B, sink_rows, Hkv, D]
+    const int32_t* key_pos0;
+    int sink_rows;
     float sl2;              // softmax scale * log2(e)
     float scale;
 };
@@ -228,19 +233,26 @@ struct PrefillSmem {
 struct WorkItem {
     int valid, seq_start, seq_len, m_tile, pair;
     int k_start;  // first packed key token of the sequence (= seq_start for self attention; sequence index when paged)
-    int k_off;    // position of the sequence's first query inside its sequence: len_k - len_q (0 for self attention)
+    int k_off;    // index of the sequence's first query among its (local) keys: len_k - len_q (0 for self attention)
+    int full;     // this item runs full causal attention (per sequence in a mixed batch)
+    int n_sink;   // sink keys among the local keys (context-parallel: n_sink - key_pos0, clamped; else n_sink)
+    int s_rem;    // context-parallel: sink keys that come from the separate sink buffer, min(n_sink, key_pos0)
+    int b;        // context-parallel: sequence index (row of the sink buffer)
 };
 
 // kMode 0: self attention.  1: chunked prefill, the queries are the last len_q tokens of a longer key sequence
 // (separate packing of the keys).  2: the same with keys and values in pages addressed through a block table.
+// 3: context-parallel prefill, mode 1 with the local keys starting at position key_pos0[b] of their sequence and the
+// sink keys before that position read from a separate buffer (tm_sk, tm_sv) as leading key tiles of the item.
 // The self-attention instance compiles the offsets away.
 template <int D, int kMode>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+               const __grid_constant__ CUtensorMap tm_sk, const __grid_constant__ CUtensorMap tm_sv,
                const PrefillParams p) {
     using L = PrefillSmem<D>;
-    constexpr bool kChunked = kMode >= 1, kPaged = kMode == 2;
+    constexpr bool kChunked = kMode >= 1, kPaged = kMode == 2, kCp = kMode == 3;
     constexpr int BM = kPrefillBM, BN = kPrefillBN;
     constexpr int ST = L::kStages;
     constexpr uint32_t kIdescQK = make_idesc(BM, BN, 0);
@@ -265,10 +277,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     static_assert(BAR_VC + ST == L::kNumBars, "barrier count");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + L::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile int* work_ring = reinterpret_cast<volatile int*>(tmem_slot + 4);  // 2 slots x 8 ints
+    volatile int* work_ring = reinterpret_cast<volatile int*>(tmem_slot + 4);  // 2 slots x 12 ints
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool full = p.is_full != 0;
+    const bool full_all = p.is_full != 0;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -295,7 +307,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     auto fetch_work = [&](int it, WorkItem& w, bool release) -> bool {
         const int slot = it & 1;
         if (!mbar_wait(bar(BAR_WF + slot), (uint32_t)(it >> 1) & 1u, abort_flag)) return false;
-        volatile int* d = work_ring + slot * 8;
+        volatile int* d = work_ring + slot * 12;
         w.valid = d[0];
         w.seq_start = d[1];
         w.seq_len = d[2];
@@ -303,6 +315,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         w.pair = d[4];
         w.k_start = kChunked ? d[5] : w.seq_start;
         w.k_off = kChunked ? d[6] : 0;
+        w.full = kChunked ? d[7] : (full_all ? 1 : 0);
+        w.n_sink = kCp ? d[8] : p.n_sink;
+        w.s_rem = kCp ? d[9] : 0;
+        w.b = kCp ? d[10] : 0;
         if (release) mbar_arrive(bar(BAR_WE + slot));
         return true;
     };
@@ -317,6 +333,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (lane == 0) {
             if (p.cu_seqlens[0] != 0 || p.cu_seqlens[p.B] != p.T) record_device_error(SWAA_ERR_BAD_SEQLENS);
             int b = p.B, acc = 0, cur_nt = 0, cur_s = 0, cur_len = 0, cur_ks = 0, cur_off = 0;
+            int cur_full = full_all ? 1 : 0, cur_sink = p.n_sink, cur_srem = 0;
             auto next_seq = [&]() {
                 acc += cur_nt;
                 --b;
@@ -346,7 +363,19 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         }
                         cur_ks = ks;
                         cur_off = ke - ks - len;
+                        if (kCp) {
+                            // the local keys start at position p0: the sink keys before it come from the sink buffer,
+                            // and the window of the first query must not reach below p0 (halo of window - 1 keys)
+                            const int p0 = p.key_pos0[b];
+                            if (p0 < 0 || (p0 > 0 && cur_off < p.window - 1) || (p0 > 0 && p.n_sink > p.sink_rows)) {
+                                record_device_error(SWAA_ERR_BAD_SEQLENS);
+                                len = 0;
+                            }
+                            cur_srem = p0 < p.n_sink ? max(p0, 0) : p.n_sink;
+                            cur_sink = p.n_sink - cur_srem;
+                        }
                     }
+                    if (kChunked && p.is_full_seq != nullptr) cur_full = p.is_full_seq[b] != 0 ? 1 : 0;
                     cur_s = s0;
                     cur_len = len;
                     cur_nt = (len + BM - 1) / BM;
@@ -360,7 +389,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 while (b >= 0 && tile_id >= (long long)acc + cur_nt) next_seq();
                 const int slot = it & 1;
                 if (!mbar_wait(bar(BAR_WE + slot), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag)) break;
-                volatile int* d = work_ring + slot * 8;
+                volatile int* d = work_ring + slot * 12;
                 d[0] = b >= 0 ? 1 : 0;
                 d[1] = cur_s;
                 d[2] = cur_len;
@@ -369,6 +398,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (kChunked) {
                     d[5] = cur_ks;
                     d[6] = cur_off;
+                    d[7] = cur_full;
+                }
+                if (kCp) {
+                    d[8] = cur_sink;
+                    d[9] = cur_srem;
+                    d[10] = b;
                 }
                 mbar_arrive(bar(BAR_WF + slot));
                 if (b < 0) break;
@@ -389,8 +424,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
                 const bool hasB = (hA + 1) < (hk + 1) * p.G;
                 const int i0 = w.m_tile * BM, i1 = min(w.seq_len, i0 + BM) - 1;
-                const TileRange tr = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, p.n_sink, full);
-                const int nt = tr.count();
+                const TileRange tr = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, w.n_sink, w.full != 0);
+                const int n_rem = kCp ? (w.s_rem + BN - 1) / BN : 0;  // leading tiles from the sink buffer
+                const int nt = n_rem + tr.count();
                 // Q tiles of both sides (the previous item's last QK must have retired)
                 ok = mbar_wait(bar(BAR_QE), ((uint32_t)items & 1u) ^ 1u, abort_flag);
                 if (!ok) break;
@@ -407,7 +443,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 for (int n = 0; n < nt; ++n, ++g) {
                     const int s = g % ST;
                     const uint32_t ph = (uint32_t)(g / ST) & 1u;
-                    const int kt = tr.tile(n) * BN;  // first key of the tile, counted inside the sequence
+                    const bool remote = kCp && n < n_rem;
+                    const int kt = remote ? n * BN : tr.tile(n - n_rem) * BN;  // first key of the tile, counted inside the (local) keys
                     int tk = w.k_start + kt, page = 0;  // packed token index, or (row in page, page) when paged
                     if (kPaged) {
                         page = __ldg(p.block_table + (size_t)w.k_start * p.max_blocks + kt / p.page_size);
@@ -423,6 +460,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                     for (int pn = 0; pn < L::kPanels; ++pn) {
                         if (kPaged) tma_load_4d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, page, bar(BAR_KF + s));
+                        else if (remote) tma_load_4d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_sk, pn * 64, hk, kt, w.b, bar(BAR_KF + s));
                         else tma_load_3d(sK + s * L::kTileBytes + pn * L::kPanelBytes, &tm_k, pn * 64, hk, tk, bar(BAR_KF + s));
                     }
                     ok = mbar_wait(bar(BAR_VE + s), ph ^ 1u, abort_flag);
@@ -434,6 +472,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
                     for (int pn = 0; pn < L::kPanels; ++pn) {
                         if (kPaged) tma_load_4d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, page, bar(BAR_VF + s));
+                        else if (remote) tma_load_4d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_sv, pn * 64, hk, kt, w.b, bar(BAR_VF + s));
                         else tma_load_3d(sV + s * L::kTileBytes + pn * L::kPanelBytes, &tm_v, pn * 64, hk, tk, bar(BAR_VF + s));
                     }
                     if (kPaged) {
@@ -524,8 +563,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int hA = hk * p.G + 2 * (w.pair - hk * p.pairs_per_kv);
                 const bool hasB = (hA + 1) < (hk + 1) * p.G;
                 const int i0 = w.m_tile * BM, i1 = min(w.seq_len, i0 + BM) - 1;
-                const TileRange trng = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, p.n_sink, full);
-                const int nt = trng.count();
+                const TileRange trng = tile_range(i0 + w.k_off, i1 + w.k_off, BN, p.window, w.n_sink, w.full != 0);
+                const int nt = (kCp ? (w.s_rem + BN - 1) / BN : 0) + trng.count();
                 ok = mbar_wait(bar(BAR_QF), (uint32_t)items & 1u, abort_flag) &&
                      mbar_wait(bar(BAR_KF + g % ST), (uint32_t)(g / ST) & 1u, abort_flag);
                 if (!ok) break;
@@ -628,14 +667,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const int q0 = w.m_tile * BM;    // first query of the tile, counted inside the sequence's queries
             const int iq = q0 + row;         // this thread's query, same counting
             const int i0 = q0 + w.k_off, i1 = min(seq_len, q0 + BM) - 1 + w.k_off;  // positions inside the sequence
-            const TileRange tr = tile_range(i0, i1, BN, p.window, p.n_sink, full);
-            const int nt = tr.count();
-            const int i = iq + w.k_off;      // position of this thread's query inside its sequence
+            const bool full = w.full != 0;
+            const TileRange tr = tile_range(i0, i1, BN, p.window, w.n_sink, full);
+            const int n_rem = kCp ? (w.s_rem + BN - 1) / BN : 0;  // leading tiles from the sink buffer
+            const int nt = n_rem + tr.count();
+            const int i = iq + w.k_off;      // index of this thread's query among the (local) keys of its sequence
             const int h = hA + side;
             float m_used = -INFINITY, l_sum = 0.f;
             for (int n = 0; n < nt; ++n, ++gs) {
-                const int j0 = tr.tile(n) * BN;
-                const bool need_mask = tile_needs_mask(i0, i1, j0, j0 + BN - 1, p.window, p.n_sink, full);
+                // a tile from the sink buffer holds positions before every local key: all rows see exactly its keys
+                // below s_rem; no window or causal edge runs through it
+                const bool remote = kCp && n < n_rem;
+                const int j0 = remote ? n * BN : tr.tile(n - n_rem) * BN;
+                const bool need_mask = remote ? (w.s_rem - j0 < BN)
+                                              : tile_needs_mask(i0, i1, j0, j0 + BN - 1, p.window, w.n_sink, full);
                 ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SF + side), (uint32_t)gs & 1u, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
@@ -649,9 +694,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (need_mask) {
                     // Bit b of vis[cc] <=> column c = 32*cc + b of this tile is visible to this row:
                     //   c <= dc  and  ( c > wl  or  c < sk ).
-                    const int dc = i - j0;
-                    const int wl = full ? -1 : dc - p.window;
-                    const int sk = full ? 0 : p.n_sink - j0;
+                    const int dc = remote ? (1 << 20) : i - j0;
+                    const int wl = remote ? (1 << 20) : (full ? -1 : dc - p.window);
+                    const int sk = remote ? w.s_rem - j0 : (full ? 0 : w.n_sink - j0);
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         const int d = dc - 32 * cc, wd = wl - 32 * cc, sn = sk - 32 * cc;

@@ -140,3 +140,47 @@ def test_lazy_ratio_matches_oracle():
         got = ratio.cpu().numpy()
         assert np.abs(got - ref).max() <= 5e-3, (got, ref)
         assert ((ref > 0.05) & (ref < 0.999)).any()
+
+
+def test_mixed_batch_with_a_mask_policy_per_sequence():
+    """One launch serving prefill chunks under the SWA mask next to single decode tokens under full attention
+    (Fig. 1a), dense and paged keys, against the oracle's per-sequence policy."""
+    lq, lk = (130, 1, 300, 1, 64), (130, 1700, 900, 129, 64)
+    flags = [0, 1, 0, 1, 1]
+    fs = torch.tensor(flags, dtype=torch.uint8, device="cuda")
+    for Hq, Hkv, D in ((4, 2, 128), (6, 2, 64)):
+        q, k, v = make(lq, lk, Hq, Hkv, D, seed=900 + D)
+        qh, kh, vh = (inputs.to_f32_numpy(t) for t in (q, k, v))
+        for W, S in ((128, 4), (100, 7), (1, 0)):
+            Tq = sum(lq)
+            out = torch.full((Tq, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+            lse = torch.full((Hq, Tq), float("nan"), dtype=torch.float32, device="cuda")
+            swaa.swaa_prefill_chunked(q, k, v, out, _cu(lq), _cu(lk), max(lq), max(lk), W, S, False, lse=lse,
+                                      is_full_seq=fs)
+            assert swaa.last_device_status() == 0
+            ref = oracle.prefill_chunked(qh, kh, vh, _cu(lq).cpu().numpy(), _cu(lk).cpu().numpy(), W, S, False,
+                                         is_full_seq=flags)
+            check_against_oracle(out, ref["out"], f"mixed batch D={D} W={W} S={S}")
+            np.testing.assert_allclose(lse.cpu().numpy().T, ref["lse"], rtol=0, atol=2e-3)
+            # the same keys scattered over pages
+            page = 128
+            blocks = [(n + page - 1) // page for n in lk]
+            num_pages = sum(blocks) + 2
+            perm = np.random.default_rng(5).permutation(num_pages)
+            kp = torch.full((num_pages, page, Hkv, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+            vp = torch.full_like(kp, float("nan"))
+            bt = np.full((len(lk), max(blocks)), -1, dtype=np.int32)
+            cuk = np.concatenate([[0], np.cumsum(lk)])
+            nxt = 0
+            for b, n in enumerate(lk):
+                for blk in range(blocks[b]):
+                    pg = int(perm[nxt]); nxt += 1
+                    bt[b, blk] = pg
+                    m = min(page, n - blk * page)
+                    kp[pg, :m] = k[cuk[b] + blk * page:cuk[b] + blk * page + m]
+                    vp[pg, :m] = v[cuk[b] + blk * page:cuk[b] + blk * page + m]
+            out2 = torch.full_like(out, float("nan"))
+            swaa.swaa_prefill_paged(q, kp, vp, out2, _cu(lq), torch.tensor(lk, dtype=torch.int32, device="cuda"),
+                                    torch.as_tensor(bt, device="cuda"), max(lq), W, S, False, is_full_seq=fs)
+            assert swaa.last_device_status() == 0
+            check_against_oracle(out2, ref["out"], f"mixed paged batch D={D} W={W} S={S}")
