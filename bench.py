@@ -217,6 +217,88 @@ def time_prefill_case(swaa, torch, flush_l2, stream, peaks, cfg, is_full, reps, 
             "frac_of_nominal_2250": tf / 2250.0, "us_per_1k_tokens": 1e3 * st["median"] / (sum(cfg.seqlens) / 1024.0)}
 
 
+def gather_decode_partials(part, world):
+    """The one exchange of a decode whose cache is cut along the context: every rank contributes its partial
+    results [B, Hq, D + 2] (float32) and receives all of them as [world, B, Hq, D + 2], rank-major, ready for
+    swaa_decode_combine.  B * Hq * (D + 2) floats per rank (266 KB at workload 4)."""
+    import torch
+
+    if world == 1:
+        return part.unsqueeze(0).contiguous()
+    import torch.distributed as dist
+
+    out = torch.empty((world,) + tuple(part.shape), dtype=part.dtype, device=part.device)
+    # concatenation along the first dimension: rank r's partials land in rows [r * B, (r + 1) * B)
+    dist.all_gather_into_tensor(out.view((world * part.shape[0],) + tuple(part.shape[1:])), part.contiguous())
+    return out
+
+
+def run_decode_split(args, rank, local_rank, world):
+    """Decode workload 4 with the cache cut along the context over the ranks (strong scaling: the job is one decode
+    step of the whole batch).  Rank r holds positions [r * Lmax / N, (r + 1) * Lmax / N) of every sequence; a step is
+    swaa_decode_partial on the shard, the gather of the partials, swaa_decode_combine.  With one rank the shards of an
+    N-way cut (--shards) are run one after another on the same GPU, which gives kernel times but no exchange."""
+    import torch
+
+    import paper_2512_10411_b200 as swaa
+    from paper_2512_10411_b200 import inputs
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    dcfg = inputs.cfg_decode()
+    P = world if world > 1 else max(1, args.shards)
+    Lsh = dcfg.Lmax // P
+    mine = [rank] if world > 1 else list(range(P))
+    q, kc, vc, sl = inputs.make_decode_inputs(dcfg, dev)
+    shards = [(kc[:, r * Lsh:(r + 1) * Lsh].contiguous(), vc[:, r * Lsh:(r + 1) * Lsh].contiguous(), r * Lsh) for r in mine]
+    del kc, vc
+    out = torch.empty_like(q)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_rd = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    results = {}
+    for full in (True, False):
+        ws = torch.empty(swaa.decode_partial_workspace_size(dcfg.B, dcfg.Hq, dcfg.Hkv, dcfg.D, Lsh, dcfg.window, dcfg.n_sink,
+                                                            full), dtype=torch.uint8, device=dev)
+        parts = torch.empty((len(mine), dcfg.B, dcfg.Hq, dcfg.D + 2), dtype=torch.float32, device=dev)
+        times = []
+        for it in range(max(args.warmup, 3) + args.steps):
+            flush.zero_()
+            flush_rd.sum()
+            if world > 1:
+                dist.barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i, (ks, vs, p0) in enumerate(shards):
+                swaa.swaa_decode_partial(q, ks, vs, parts[i], sl, p0, dcfg.window, dcfg.n_sink, full, ws)
+            allp = gather_decode_partials(parts[0], world) if world > 1 else parts
+            swaa.swaa_decode_combine(allp, out)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if it >= max(args.warmup, 3):
+                times.append(a.elapsed_time(b))
+        assert swaa.last_device_status() == 0
+        med = max_over_ranks([stats_ms(times)["median"]], world, dev)[0]
+        nbytes = float(dcfg.B) * (dcfg.Lmax if full else dcfg.window + dcfg.n_sink) * dcfg.Hkv * dcfg.D * 4
+        results["fa" if full else "swa"] = {"us_per_step": 1e3 * med, "gbs": nbytes / (med * 1e-3) / 1e9, "bytes": nbytes}
+    if rank == 0:
+        print(json.dumps({"metric": "decode_split_hbm_gbs", "value": results["fa"]["gbs"], "unit": "GB/s", "n_gpus": world,
+                          "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": results["fa"]["us_per_step"] / 1e3,
+                          "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+                          "data": "synthetic",
+                          "config": {"workload": f"cfg4 decode B=16 Lcache=65536 cut along the context into {P} shards"
+                                                 + ("" if world > 1 else " run one after another on one GPU (no exchange)"),
+                                     "l2": "flushed before every step"},
+                          "decode_split": results, "hbm_peak_gbs": peaks["hbm_gbs"]}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def whole_job_value(units_per_rank, n_ranks, seconds):
     """Throughput of the whole job: the units all ranks processed over the slowest rank's time."""
     return n_ranks * units_per_rank / seconds
@@ -734,6 +816,10 @@ def main():
                     help="run three launches of one kernel only (for ncu) and exit")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the workloads outside the timed step (workloads 1, 3, 5 and the L sweep)")
+    ap.add_argument("--decode-split", action="store_true",
+                    help="decode workload 4 with the cache cut along the context over the ranks (or, on one GPU, over "
+                         "--shards shards run in sequence) and exit")
+    ap.add_argument("--shards", type=int, default=4)
     ap.add_argument("--sweep", action="store_true",
                     help="time swaa_prefill on the other workloads and the L / W / n_sink sweeps (one GPU) and exit")
     args = ap.parse_args()
@@ -746,7 +832,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
+    if args.decode_split:
+        run_decode_split(args, rank, local_rank, world)
+    elif args.impl == "reference":
         run_reference(args, rank)
     else:
         run_ours(args, rank, local_rank, world)

@@ -245,6 +245,37 @@ int swaa_decode_paged(const void* q, const void* kpages, const void* vpages, voi
                       void* stream);
 
 /*
+ * Decode with the KV cache cut along the context (App. A: under FA decode the cache of the whole context must be
+ * retained, which is what makes spreading it over several devices attractive; Sec. 3.1.1).  A participant holds, for
+ * every sequence, the entries at positions key_pos0 .. key_pos0 + Lshard - 1 and computes the partial result of
+ * every (sequence, head) row over the visible keys it holds; the partials of all participants (B * Hq * (D + 2)
+ * floats each: gather them with any collective or copy) are merged by swaa_decode_combine.  The mask is evaluated
+ * on positions of the whole sequence, so the result equals swaa_decode on the uncut cache.
+ *
+ *   kshard, vshard  device, [B, Lshard, Hkv, D] bf16; entry at position p of sequence b in row p - key_pos0.
+ *                   Rows that lie past a sequence's length are never used, whatever they hold.
+ *   seqlens         device, int32 [B]: TOTAL number of valid entries of each sequence (>= 1) including the current
+ *                   token; the query sits at position seqlens[b] - 1.  A value < 1 is reported as
+ *                   SWAA_ERR_BAD_SEQLENS through the status word.
+ *   partial_out     device, float32 [B, Hq, D + 2]: (m, l, o[0..D)) with m = largest visible scaled score held by
+ *                   this participant (natural-log units), l = sum of exp(score - m), o = sum of exp(score - m) * v.
+ *                   A participant that holds no visible key of a row writes (-inf, 0, 0...).
+ *   workspace       at least swaa_decode_partial_workspace_size(...) bytes, 256-byte aligned, uninitialised.
+ * Other arguments and status codes as for swaa_decode (same kernel; the split-K merge across thread blocks happens
+ * inside the launch as usual and produces the participant's partial).
+ *
+ * swaa_decode_combine: partials device, float32 [P, B, Hq, D + 2] (participant-major); out device, [B, Hq, D] bf16 =
+ * sum_s e^(m_s - M) o_s / sum_s e^(m_s - M) l_s with M = max_s m_s over the non-empty partials (zeros when all are
+ * empty).
+ */
+size_t swaa_decode_partial_workspace_size(int B, int Hq, int Hkv, int D, int Lshard, int window, int n_sink,
+                                          int is_full);
+int swaa_decode_partial(const void* q, const void* kshard, const void* vshard, float* partial_out,
+                        const int32_t* seqlens, int B, int Lshard, int key_pos0, int Hq, int Hkv, int D, int window,
+                        int n_sink, int is_full, float scale, void* workspace, size_t workspace_bytes, void* stream);
+int swaa_decode_combine(const float* partials, int P, int B, int Hq, int D, void* out, void* stream);
+
+/*
  * Allocation-free decode.  (The paper has no counterpart to this call; it exists for integration.)
  *
  * Same computation and arguments as swaa_decode, but the split-K scratch lives in a fixed array inside

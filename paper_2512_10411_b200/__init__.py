@@ -22,6 +22,9 @@ from .binding import (  # noqa: F401
     status_str,
     swaa_decode,
     swaa_decode_paged,
+    swaa_decode_partial,
+    swaa_decode_combine,
+    decode_partial_workspace_size,
     decode_paged_workspace_size,
     swaa_decode_static,
     DECODE_STATIC_SCRATCH_BYTES,

@@ -100,6 +100,12 @@ def load_library():
     lib.swaa_decode_paged_workspace_size.restype = ctypes.c_size_t
     lib.swaa_decode_paged.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
     lib.swaa_decode_paged.restype = ci
+    lib.swaa_decode_partial_workspace_size.argtypes = [ci] * 8
+    lib.swaa_decode_partial_workspace_size.restype = ctypes.c_size_t
+    lib.swaa_decode_partial.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp, ctypes.c_size_t, vp]
+    lib.swaa_decode_partial.restype = ci
+    lib.swaa_decode_combine.argtypes = [vp, ci, ci, ci, ci, vp, vp]
+    lib.swaa_decode_combine.restype = ci
     lib.swaa_decode_static.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, cf, vp]
     lib.swaa_decode_static.restype = ci
     lib.swaa_schedule_is_full.argtypes = [ctypes.POINTER(_Policy), ci, ci]
@@ -385,6 +391,44 @@ def swaa_decode_paged(q, kpages, vpages, out, block_table, seqlens, window: int,
                                _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
     if rc != SWAA_OK:
         raise SwaaError(rc, "swaa_decode_paged")
+
+
+def decode_partial_workspace_size(B, Hq, Hkv, D, Lshard, window, n_sink, is_full) -> int:
+    """Forwards to C swaa_decode_partial_workspace_size (bytes)."""
+    return int(load_library().swaa_decode_partial_workspace_size(B, Hq, Hkv, D, int(Lshard), int(window), int(n_sink),
+                                                                 int(bool(is_full))))
+
+
+def swaa_decode_partial(q, kshard, vshard, partial_out, seqlens, key_pos0: int, window: int, n_sink: int, is_full: bool,
+                        workspace, scale: float = 0.0, stream=None) -> None:
+    """Forwards to C swaa_decode_partial.  q [B,Hq,D]; kshard, vshard [B,Lshard,Hkv,D] bf16 holding positions key_pos0..;
+    partial_out f32 [B,Hq,D+2]; seqlens int32 [B] (total lengths)."""
+    lib = load_library()
+    B, Hq, D = q.shape
+    _, Lshard, Hkv, _ = kshard.shape
+    if tuple(kshard.shape) != (B, Lshard, Hkv, D) or tuple(vshard.shape) != (B, Lshard, Hkv, D) \
+            or tuple(partial_out.shape) != (B, Hq, D + 2) or seqlens.numel() != B:
+        raise ValueError("swaa_decode_partial: inconsistent tensor shapes")
+    bf = torch.bfloat16
+    rc = lib.swaa_decode_partial(_dev_ptr(q, bf, "q"), _dev_ptr(kshard, bf, "kshard"), _dev_ptr(vshard, bf, "vshard"),
+                                 _dev_ptr(partial_out, torch.float32, "partial_out"),
+                                 _dev_ptr(seqlens, torch.int32, "seqlens"), B, Lshard, int(key_pos0), Hq, Hkv, D,
+                                 int(window), int(n_sink), int(bool(is_full)), float(scale),
+                                 _dev_ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_decode_partial")
+
+
+def swaa_decode_combine(partials, out, stream=None) -> None:
+    """Forwards to C swaa_decode_combine.  partials f32 [P,B,Hq,D+2]; out bf16 [B,Hq,D]."""
+    lib = load_library()
+    P, B, Hq, D2 = partials.shape
+    if tuple(out.shape) != (B, Hq, D2 - 2):
+        raise ValueError("swaa_decode_combine: out must be [B, Hq, D]")
+    rc = lib.swaa_decode_combine(_dev_ptr(partials, torch.float32, "partials"), P, B, Hq, D2 - 2,
+                                 _dev_ptr(out, torch.bfloat16, "out"), _stream_ptr(stream))
+    if rc != SWAA_OK:
+        raise SwaaError(rc, "swaa_decode_combine")
 
 
 def trimmed_cache_slot(pos: int, window: int, n_sink: int) -> int:

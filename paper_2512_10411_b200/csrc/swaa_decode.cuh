@@ -49,6 +49,11 @@ struct DecodeParams {
     // paged cache only: entry j of sequence b lives in page block_table[b * max_blocks + j / page_size]
     const int32_t* block_table;
     int max_blocks, page_tiles /* page_size / 64 */, num_pages;
+    // one shard of a cache cut along the context (kShard): the buffers hold positions pos0 .. pos0 + Lmax - 1 of every
+    // sequence, seqlens are total lengths, and every row's result leaves as a partial (max, sum, unnormalised O)
+    int pos0;
+    float scale;      // softmax scale (natural-log units of the exported maximum)
+    float* part_out;  // [B, Hq, D + 2]
 };
 
 constexpr int kDecodeTileKeys = 64;
@@ -75,42 +80,77 @@ struct DecodeSmem {
     static constexpr int kDynamicBytes = kBytes + 1024;  // room to align the base to 1024 B
 };
 
-// Visible part of one sequence's cache, in tiles.
+// Visible part of one sequence's cache, in tiles, as row ranges of the buffer the kernel reads.
 struct SeqGeom {
     int len;  // valid entries (0 when seqlens[b] is out of range)
-    int lo;   // first window key
-    int ns;   // sink keys that lie before the window
+    int sb;   // first sink row (0 unless the buffer is a shard that starts inside the sinks)
+    int se;   // end of the sink rows that lie before the window
     int nst;  // sink tiles
     int nt;   // tiles per item
-    int w0;   // first key of the first window tile: lo (dense cache), or lo rounded down to a tile (paged cache)
+    int wb;   // first window row
+    int we;   // end of the window rows (the sequence's last valid entry + 1)
+    int w0;   // first row of the first window tile: wb (dense cache), or wb rounded down to a tile (paged cache)
 };
 
 // With `aligned` the window tiles start on multiples of the tile size, so that no tile straddles a page of
-// a paged cache; the keys before `lo` in the first window tile are then masked like those past `len`.
+// a paged cache; the keys before the window in the first window tile are then masked like those past the end.
 __host__ __device__ inline SeqGeom decode_seq_geom(int len, int Lmax, int window, int n_sink, int is_full,
                                                    bool aligned = false) {
     SeqGeom s;
     if (len < 1 || len > Lmax) {
-        s.len = s.lo = s.ns = s.nst = s.nt = s.w0 = 0;
+        s.len = s.sb = s.se = s.nst = s.nt = s.wb = s.we = s.w0 = 0;
         return s;
     }
     s.len = len;
-    s.lo = is_full ? 0 : (len > window ? len - window : 0);
-    s.ns = is_full ? 0 : (n_sink < s.lo ? n_sink : s.lo);
-    s.nst = (s.ns + kDecodeTileKeys - 1) / kDecodeTileKeys;
-    s.w0 = aligned ? s.lo / kDecodeTileKeys * kDecodeTileKeys : s.lo;
+    s.wb = is_full ? 0 : (len > window ? len - window : 0);
+    s.we = len;
+    s.sb = 0;
+    s.se = is_full ? 0 : (n_sink < s.wb ? n_sink : s.wb);
+    s.nst = (s.se + kDecodeTileKeys - 1) / kDecodeTileKeys;
+    s.w0 = aligned ? s.wb / kDecodeTileKeys * kDecodeTileKeys : s.wb;
     s.nt = s.nst + (len - s.w0 + kDecodeTileKeys - 1) / kDecodeTileKeys;
     return s;
 }
 
+// The same for a shard that holds positions [pos0, pos0 + rows) of a sequence of `len` tokens in total: the visible
+// positions (sinks before the window, then the window ending at the query at len - 1) cut to what the shard holds
+// and moved to its row numbers.  A shard may hold no visible key at all (nt == 0 with len >= 1).
+__host__ __device__ inline SeqGeom decode_shard_geom(int len, int rows, int pos0, int window, int n_sink, int is_full) {
+    SeqGeom s;
+    s.len = s.sb = s.se = s.nst = s.nt = s.wb = s.we = s.w0 = 0;
+    if (len < 1) return s;
+    s.len = len;
+    const long long end = (long long)pos0 + rows;  // first position past the shard
+    const int lo = is_full ? 0 : (len > window ? len - window : 0);
+    const int ns = is_full ? 0 : (n_sink < lo ? n_sink : lo);
+    const long long sb = pos0 < ns ? pos0 : ns, se = end < ns ? end : ns;          // sinks in [pos0, end)
+    const long long wb = lo > pos0 ? lo : pos0, we = end < len ? end : len;        // window in [pos0, end)
+    if (se > sb) {
+        s.sb = (int)(sb - pos0);
+        s.se = (int)(se - pos0);
+    }
+    if (we > wb) {
+        s.wb = (int)(wb - pos0);
+        s.we = (int)(we - pos0);
+    }
+    s.w0 = s.wb;
+    s.nst = (s.se - s.sb + kDecodeTileKeys - 1) / kDecodeTileKeys;
+    s.nt = s.nst + (s.we - s.w0 + kDecodeTileKeys - 1) / kDecodeTileKeys;
+    return s;
+}
+
 // Position in the global tile list; every role of a block walks the same positions.
-template <bool kPaged>
+template <bool kPaged, bool kShard>
 struct DecodeWalker {
     int b, hv, ti;
     SeqGeom s;
+    static __device__ __forceinline__ SeqGeom geom(const DecodeParams& p, int b) {
+        if (kShard) return decode_shard_geom(__ldg(p.seqlens + b), p.Lmax, p.pos0, p.window, p.n_sink, p.is_full);
+        return decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full, kPaged);
+    }
     __device__ __forceinline__ void seek(const DecodeParams& p, int b0, long long off) {
         b = b0;
-        s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full, kPaged);
+        s = geom(p, b);
         hv = (int)(off / s.nt);
         ti = (int)(off - (long long)hv * s.nt);
     }
@@ -120,18 +160,20 @@ struct DecodeWalker {
         if (++hv < p.IPB) return;
         hv = 0;
         while (++b < p.B) {
-            s = decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full, kPaged);
+            s = geom(p, b);
             if (s.nt > 0) return;
         }
         s.nt = 0;  // past the last sequence
     }
-    __device__ __forceinline__ int key0() const { return ti < s.nst ? ti * kDecodeTileKeys : s.w0 + (ti - s.nst) * kDecodeTileKeys; }
+    __device__ __forceinline__ int key0() const {
+        return ti < s.nst ? s.sb + ti * kDecodeTileKeys : s.w0 + (ti - s.nst) * kDecodeTileKeys;
+    }
     // rows [vbegin, vend) of this tile hold visible keys; vbegin > 0 only in the first window tile of a paged cache
     __device__ __forceinline__ int vend() const {
-        const int left = ti < s.nst ? s.ns - ti * kDecodeTileKeys : s.len - key0();
+        const int left = (ti < s.nst ? s.se : s.we) - key0();
         return left < kDecodeTileKeys ? left : kDecodeTileKeys;
     }
-    __device__ __forceinline__ int vbegin() const { return (kPaged && ti == s.nst) ? s.lo - s.w0 : 0; }
+    __device__ __forceinline__ int vbegin() const { return (kPaged && ti == s.nst) ? s.wb - s.w0 : 0; }
 };
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -152,7 +194,7 @@ __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumerThreads) : "memory");
 }
 
-template <int D, int NH, bool kPaged>
+template <int D, int NH, bool kPaged, bool kShard = false>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
               const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16, const DecodeParams p) {
@@ -200,14 +242,20 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     }
 
     // ---- where does this block's run of the global tile list start?  (scan of tiles per sequence)
-    auto tiles_of = [&](int b) -> long long {
-        return (long long)decode_seq_geom(__ldg(p.seqlens + b), p.Lmax, p.window, p.n_sink, p.is_full, kPaged).nt * p.IPB;
-    };
-    auto zero_fill_bad = [&](int b) {  // a sequence without tiles: report it, zero its output rows (one block does)
-        record_device_error(SWAA_ERR_BAD_SEQLENS);
+    auto tiles_of = [&](int b) -> long long { return (long long)DecodeWalker<kPaged, kShard>::geom(p, b).nt * p.IPB; };
+    // A sequence without tiles.  Dense / paged cache: its length is out of range; report it and zero its output
+    // rows.  Shard: also what a shard that holds none of the sequence's visible keys looks like; its rows get the
+    // empty partial (-inf, 0, 0...), and only a length < 1 is an error.  One block does the stores.
+    auto zero_fill_bad = [&](int b) {
+        if (!kShard || __ldg(p.seqlens + b) < 1) record_device_error(SWAA_ERR_BAD_SEQLENS);
         if (b % ncta == cta) {
-            uint4* o = reinterpret_cast<uint4*>(p.out + (size_t)b * p.Hq * D);
-            for (int i = 0; i < p.Hq * D / 8; ++i) o[i] = make_uint4(0, 0, 0, 0);
+            if (kShard) {
+                float* o = p.part_out + (size_t)b * p.Hq * (D + 2);
+                for (int i = 0; i < p.Hq * (D + 2); ++i) o[i] = (i % (D + 2) == 0) ? -INFINITY : 0.f;
+            } else {
+                uint4* o = reinterpret_cast<uint4*>(p.out + (size_t)b * p.Hq * D);
+                for (int i = 0; i < p.Hq * D / 8; ++i) o[i] = make_uint4(0, 0, 0, 0);
+            }
         }
     };
     long long total, tpc, t0, t1, off0 = 0;
@@ -297,7 +345,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     if (warp == kDecodeConsumerWarps) {
         // =========================================================================== TMA producer
         if (lane == 0) {
-            DecodeWalker<kPaged> w;
+            DecodeWalker<kPaged, kShard> w;
             w.seek(p, b0, off0);
             bool ok = true;
             int n = 0, s = 0;
@@ -359,7 +407,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const int vrow = 16 * warp + (lane & 7) + 8 * (lane >> 4);        // V: matrices (channels lo/hi) x (keys lo/hi)
     const int vchk = (lane >> 3) & 1;
 
-    DecodeWalker<kPaged> w;
+    DecodeWalker<kPaged, kShard> w;
     w.seek(p, b0, off0);
     bool ok = true;
     bool first_seg = true;
@@ -534,7 +582,16 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
             if (!ok) continue;
             if (complete) {
-                p.out[((size_t)b * p.Hq + h0 + hh) * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+                if (kShard) {  // the row's result leaves as a partial: (max in natural-log units, sum, unnormalised O)
+                    float* po = p.part_out + ((size_t)b * p.Hq + h0 + hh) * (D + 2);
+                    po[2 + d] = num;
+                    if (d == 0) {
+                        po[0] = M * p.scale;
+                        po[1] = den;
+                    }
+                } else {
+                    p.out[((size_t)b * p.Hq + h0 + hh) * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+                }
             } else {
                 my_part[hh * (D + 2) + 2 + d] = num;
                 if (d == 0) {
@@ -609,13 +666,50 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                             num += wgt * __ldcg(pp + 2 + d);
                         }
                     }
-                    p.out[((size_t)b * p.Hq + h0 + hh) * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+                    if (kShard) {
+                        float* po = p.part_out + ((size_t)b * p.Hq + h0 + hh) * (D + 2);
+                        po[2 + d] = num;
+                        if (d == 0) {
+                            po[0] = M * p.scale;
+                            po[1] = den;
+                        }
+                    } else {
+                        p.out[((size_t)b * p.Hq + h0 + hh) * D + d] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+                    }
                 }
             }
         }
         consumer_sync();  // the merge buffers are free for the next segment
         first_seg = false;
     }
+}
+
+// Log-sum-exp combine of P partial results per (sequence, head) row: one warp per row, lanes over the channels.
+// part [P][rows][D + 2] = (max in natural-log units, sum, unnormalised O); empty partials (sum == 0) are skipped; a
+// row without any non-empty partial gives zeros.
+template <int D>
+__global__ void decode_combine_kernel(const float* __restrict__ part, int P, int rows, __nv_bfloat16* __restrict__ out) {
+    const int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    float M = -INFINITY;
+    for (int s = 0; s < P; ++s) {
+        const float* pr = part + ((size_t)s * rows + row) * (D + 2);
+        if (pr[1] > 0.f) M = fmaxf(M, pr[0]);
+    }
+    float den = 0.f, acc[D / 32];
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+    for (int s = 0; s < P; ++s) {
+        const float* pr = part + ((size_t)s * rows + row) * (D + 2);
+        if (!(pr[1] > 0.f)) continue;
+        const float w = __expf(pr[0] - M);
+        den += w * pr[1];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) acc[c] += w * pr[2 + c * 32 + lane];
+    }
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) out[(size_t)row * D + c * 32 + lane] = __float2bfloat16_rn(acc[c] * inv);
 }
 
 }  // namespace swaa

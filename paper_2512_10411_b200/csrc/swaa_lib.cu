@@ -59,15 +59,17 @@ struct DecodePlan {
 // One block per SM, fewer when the whole problem has fewer tiles than that.  Depends only on the
 // shape arguments and the SM count (sequence lengths are read on the device).
 static DecodePlan plan_decode(int B, int Hq, int Hkv, int D, int Lmax, int window, int n_sink, int is_full,
-                              int sm_count, bool paged = false) {
+                              int sm_count, bool paged = false, bool shard = false) {
     DecodePlan pl;
     const int G = Hq / Hkv;
     pl.NH = G > 8 ? 2 : 1;
     const int HC = 8 * pl.NH;
     pl.HG = (G + HC - 1) / HC;
     const SeqGeom longest = decode_seq_geom(Lmax, Lmax, window, n_sink, is_full, paged);
-    // upper bound on the tiles of one item: a shorter sequence may have one more (ragged) sink tile
-    const long long tiles_ub = (long long)B * Hkv * pl.HG * ((long long)longest.nt + 1);
+    // upper bound on the tiles of one item: a shorter sequence may have one more (ragged) sink tile; a shard of a
+    // longer sequence at most its rows in tiles plus a ragged sink and a ragged window tile
+    const long long per_item = shard ? ((long long)Lmax + kDecodeTileKeys - 1) / kDecodeTileKeys + 2 : (long long)longest.nt + 1;
+    const long long tiles_ub = (long long)B * Hkv * pl.HG * per_item;
     long long blocks = (tiles_ub + kDecodeMinTilesPerBlock - 1) / kDecodeMinTilesPerBlock;
     const long long sms = sm_count > 0 ? sm_count : 148;
     if (blocks > sms) blocks = sms;
@@ -133,13 +135,13 @@ static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, i
     return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
-template <int D, int NH, bool kPaged>
+template <int D, int NH, bool kPaged, bool kShard = false>
 static int launch_decode(const CUtensorMap (&tm)[4], const DecodeParams& p, int blocks, cudaStream_t st) {
     using L = DecodeSmem<D, NH>;
-    if (cudaFuncSetAttribute(decode_kernel<D, NH, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(decode_kernel<D, NH, kPaged, kShard>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              L::kDynamicBytes) != cudaSuccess)
         return SWAA_ERR_CUDA;
-    decode_kernel<D, NH, kPaged><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tm[0], tm[1], tm[2], tm[3], p);
+    decode_kernel<D, NH, kPaged, kShard><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tm[0], tm[1], tm[2], tm[3], p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
@@ -171,20 +173,22 @@ namespace swaa {
 static int decode_impl(const void* q, const void* kcache, const void* vcache, void* out, const int32_t* seqlens,
                        const int32_t* block_table, int max_blocks, int num_pages, int page_size, int B, int Lmax, int Hq,
                        int Hkv, int D, int window, int n_sink, int is_full, float scale, void* workspace,
-                       size_t workspace_bytes, void* stream) {
+                       size_t workspace_bytes, void* stream, float* part_out = nullptr, int pos0 = 0) {
     const bool paged = block_table != nullptr;
+    const bool shard = part_out != nullptr;  // one shard of a cache cut along the context: `out` is not used
     int rc = check_decode_shape(B, Hq, Hkv, D, Lmax, window, n_sink, is_full);
     if (rc != SWAA_OK) return rc;
     if (B == 0) return SWAA_OK;
-    if (!q || !kcache || !vcache || !out || !seqlens) return SWAA_ERR_INVALID_ARG;
+    if (!q || !kcache || !vcache || (!out && !shard) || !seqlens) return SWAA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(kcache) || !aligned16(vcache) || !aligned16(out)) return SWAA_ERR_INVALID_ARG;
+    if (shard && (pos0 < 0 || (reinterpret_cast<uintptr_t>(part_out) & 3u) != 0)) return SWAA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) != 0 || (reinterpret_cast<uintptr_t>(block_table) & 3u) != 0)
         return SWAA_ERR_INVALID_ARG;
     DeviceInfo info;
     rc = current_device_info(&info);
     if (rc != SWAA_OK) return rc;
     if (info.cc_major != 10) return SWAA_ERR_UNSUPPORTED;
-    const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count, paged);
+    const DecodePlan pl = plan_decode(B, Hq, Hkv, D, Lmax, window, n_sink, is_full, info.sm_count, paged, shard);
     if (pl.too_large) return SWAA_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || workspace_bytes < pl.bytes)
         return SWAA_ERR_WORKSPACE;
@@ -222,6 +226,16 @@ static int decode_impl(const void* q, const void* kcache, const void* vcache, vo
     p.max_blocks = max_blocks;
     p.page_tiles = paged ? page_size / kDecodeTileKeys : 1;
     p.num_pages = num_pages;
+    p.pos0 = pos0;
+    p.scale = sc;
+    p.part_out = part_out;
+    if (shard) {
+        if (D == 128)
+            return pl.NH == 1 ? launch_decode<128, 1, false, true>(tm, p, pl.blocks, st)
+                              : launch_decode<128, 2, false, true>(tm, p, pl.blocks, st);
+        return pl.NH == 1 ? launch_decode<64, 1, false, true>(tm, p, pl.blocks, st)
+                          : launch_decode<64, 2, false, true>(tm, p, pl.blocks, st);
+    }
     if (paged) {
         if (D == 128)
             return pl.NH == 1 ? launch_decode<128, 1, true>(tm, p, pl.blocks, st)
@@ -270,6 +284,42 @@ extern "C" int swaa_decode_paged(const void* q, const void* kpages, const void* 
     return decode_impl(q, kpages, vpages, out, seqlens, block_table, max_blocks, num_pages, page_size, B,
                        max_blocks * page_size, Hq, Hkv, D, window, n_sink, is_full, scale, workspace, workspace_bytes,
                        stream);
+}
+
+// ------------------------------------------------------- decode with the cache cut along the context
+extern "C" size_t swaa_decode_partial_workspace_size(int B, int Hq, int Hkv, int D, int Lshard, int window, int n_sink,
+                                                     int is_full) {
+    if (check_decode_shape(B, Hq, Hkv, D, Lshard, window, n_sink, is_full) != SWAA_OK || B == 0) return 256;
+    DeviceInfo info;
+    if (current_device_info(&info) != SWAA_OK) info.sm_count = 148;
+    return plan_decode(B, Hq, Hkv, D, Lshard, window, n_sink, is_full, info.sm_count, false, true).bytes;
+}
+
+extern "C" int swaa_decode_partial(const void* q, const void* kshard, const void* vshard, float* partial_out,
+                                   const int32_t* seqlens, int B, int Lshard, int key_pos0, int Hq, int Hkv, int D,
+                                   int window, int n_sink, int is_full, float scale, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+    if (!partial_out) return SWAA_ERR_INVALID_ARG;
+    return decode_impl(q, kshard, vshard, nullptr, seqlens, nullptr, 0, 0, 0, B, Lshard, Hq, Hkv, D, window, n_sink,
+                       is_full, scale, workspace, workspace_bytes, stream, partial_out, key_pos0);
+}
+
+extern "C" int swaa_decode_combine(const float* partials, int P, int B, int Hq, int D, void* out, void* stream) {
+    if (P < 1 || B < 0 || Hq < 1) return SWAA_ERR_INVALID_ARG;
+    if (D != 64 && D != 128) return SWAA_ERR_UNSUPPORTED;
+    if (B == 0) return SWAA_OK;
+    if (!partials || !out || (reinterpret_cast<uintptr_t>(partials) & 3u) != 0 || (reinterpret_cast<uintptr_t>(out) & 1u) != 0)
+        return SWAA_ERR_INVALID_ARG;
+    if ((long long)B * Hq > 0x3fffffffLL) return SWAA_ERR_UNSUPPORTED;
+    const int rows = B * Hq;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const unsigned blocks = (unsigned)((rows + 3) / 4);  // four warps per block, one row each
+    if (D == 128)
+        decode_combine_kernel<128><<<blocks, 128, 0, st>>>(partials, P, rows, static_cast<__nv_bfloat16*>(out));
+    else
+        decode_combine_kernel<64><<<blocks, 128, 0, st>>>(partials, P, rows, static_cast<__nv_bfloat16*>(out));
+    launch_counter().fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
 // ----------------------------------------------------------------------------------------- prefill

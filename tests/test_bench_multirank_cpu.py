@@ -25,6 +25,35 @@ dist.destroy_process_group()
 """
 
 
+SPLIT_WORKER = r"""
+import os, sys, json
+sys.path.insert(0, os.environ["SWAA_ROOT"])
+import numpy as np, torch
+import torch.distributed as dist
+import bench, oracle
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+B, Lmax, Hq, Hkv, D, W, S = 3, 40, 4, 2, 8, 9, 3
+g = torch.Generator().manual_seed(5)
+q = torch.randn((B, Hq, D), generator=g).to(torch.bfloat16).float().numpy()
+kc = torch.randn((B, Lmax, Hkv, D), generator=g).to(torch.bfloat16).float().numpy()
+vc = torch.randn((B, Lmax, Hkv, D), generator=g).to(torch.bfloat16).float().numpy()
+sl = [40, 7, 25]                      # rank 1 holds nothing of the second sequence
+res = {}
+for full in (False, True):
+    a, b = Lmax * rank // world, Lmax * (rank + 1) // world
+    part = oracle.decode_partial(q, kc[:, a:b], vc[:, a:b], sl, a, W, S, full)["part"]
+    allp = bench.gather_decode_partials(torch.from_numpy(part), world)   # [world, B, Hq, D + 2], rank-major
+    assert tuple(allp.shape) == (world, B, Hq, D + 2)
+    got = oracle.decode_combine(allp.numpy())
+    want = oracle.decode(q, kc, vc, sl, W, S, full)["out"]
+    res[str(full)] = float(np.abs(got - want).max())
+    assert np.array_equal(allp[rank].numpy(), part)   # my own partials sit in my slot (empty ones hold -inf)
+print(json.dumps({"rank": rank, "err": res}), flush=True)
+dist.destroy_process_group()
+"""
+
+
 def _free_port():
     import socket
     with socket.socket() as sk:
@@ -60,3 +89,17 @@ def test_reference_arm_prints_from_rank_zero_only():
     d = lines[0]
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["value"] > 0
+
+
+def test_two_rank_gather_of_decode_partials(tmp_path):
+    """The one exchange of a decode whose cache is cut along the context: two gloo ranks each form the partials of
+    their shard (here with the oracle, on CPU), gather them through bench.gather_decode_partials and combine; every
+    rank gets the result of the uncut decode."""
+    script = tmp_path / "split_worker.py"
+    script.write_text(SPLIT_WORKER)
+    r = _launch([str(script)], env_extra={"OMP_NUM_THREADS": "2"})
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert sorted(d["rank"] for d in lines) == [0, 1]
+    for d in lines:
+        assert d["err"]["False"] < 1e-13 and d["err"]["True"] < 1e-13
