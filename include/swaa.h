@@ -186,11 +186,13 @@ int swaa_prefill_context_parallel(const void* q, const void* k_local, const void
  *     ratio[h] = mean over the queries of  sum_{j recent or sink} p(i, j),
  * p = softmax of scale * q.k over ALL keys j <= i (full causal attention), "recent" = the last `recent` keys
  * ending at the query, "sink" = the first n_sink keys of the sequence.  A value near 1 marks a layer that an SWA
- * mask would hardly change.  The mass is obtained from two log-sum-exp passes of the prefill kernel (windowed
- * and full) and a small reduction kernel.
+ * mask would hardly change.  The mass is obtained from two log-sum-exp passes (windowed and full) of a prefill
+ * kernel instance that forms only the row sums (no values fetched, no P V product, no output) and a small
+ * reduction kernel.
  *
  *   ratio        device, float32 [Hq]
- *   scratch_out  device, bf16 [Tq, Hq, D]; scratch_lse device, float32 [2, Hq, Tq]; both overwritten.
+ *   scratch_lse  device, float32 [2, Hq, Tq], overwritten.
+ *   v, scratch_out  not used (the probe needs no values and writes no attention output); may be NULL.
  * Other arguments, status codes and errors as for swaa_prefill_chunked (recent >= 1, n_sink >= 0).
  */
 int swaa_lazy_ratio(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_q,

@@ -317,12 +317,12 @@ def swaa_prefill_context_parallel(q, k_local, v_local, sink_k, sink_v, out, cu_s
 
 def swaa_lazy_ratio(q, k, v, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, recent: int, n_sink: int,
                     ratio, scratch_out, scratch_lse, scale: float = 0.0, stream=None) -> None:
-    """Forwards to C swaa_lazy_ratio.  q [Tq,Hq,D]; k, v [Tk,Hkv,D] bf16; ratio f32 [Hq]; scratch_out bf16 [Tq,Hq,D];
-    scratch_lse f32 [2,Hq,Tq]."""
+    """Forwards to C swaa_lazy_ratio.  q [Tq,Hq,D]; k [Tk,Hkv,D] bf16; ratio f32 [Hq]; scratch_lse f32 [2,Hq,Tq].
+    v and scratch_out are not used by the probe and may be None."""
     lib = load_library()
     Tq, Hq, D = q.shape
     Tk, Hkv = k.shape[0], k.shape[1]
-    if tuple(scratch_out.shape) != (Tq, Hq, D) or tuple(scratch_lse.shape) != (2, Hq, Tq) or tuple(ratio.shape) != (Hq,):
+    if tuple(scratch_lse.shape) != (2, Hq, Tq) or tuple(ratio.shape) != (Hq,):
         raise ValueError("swaa_lazy_ratio: inconsistent output / scratch shapes")
     B = cu_seqlens_q.numel() - 1
     bf = torch.bfloat16

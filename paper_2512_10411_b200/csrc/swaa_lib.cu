@@ -119,10 +119,55 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+// Encoded tensor maps are kept in a small host-side table keyed by everything that goes into them: a serving loop
+// calls with the same buffers and shapes step after step, and four encodings per call are a measurable part of a
+// 50 us decode step.  A tensor map holds no device state (address and geometry only), so an entry stays valid for
+// as long as its key matches, whatever happens to the memory behind it.
+struct MapKey {
+    const void* base;
+    int kind, a, b, c, d, e;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && kind == o.kind && a == o.a && b == o.b && c == o.c && d == o.d && e == o.e;
+    }
+};
+static bool cached_map(const MapKey& key, CUtensorMap* out, const CUtensorMap* store) {
+    constexpr int kSlots = 64;
+    struct Slot {
+        bool used = false;
+        MapKey key{};
+        CUtensorMap map{};
+    };
+    static std::mutex mu;
+    static Slot slots[kSlots];
+    static unsigned next = 0;
+    std::lock_guard<std::mutex> lock(mu);
+    if (store == nullptr) {
+        for (int i = 0; i < kSlots; ++i)
+            if (slots[i].used && slots[i].key == key) {
+                *out = slots[i].map;
+                return true;
+            }
+        return false;
+    }
+    Slot& s = slots[next++ % kSlots];  // oldest entry goes
+    s.used = true;
+    s.key = key;
+    s.map = *store;
+    return true;
+}
+
 // Tensor map over a bf16 cache [B, Lmax, Hkv, D]: dimensions (D, Hkv, Lmax, B) innermost first; one box
 // is [box_keys entries] x [1 head] x [64 channels] = rows of 128 bytes, written with the 128-byte swizzle.
 // Rows past Lmax are filled with zeros.
+static int make_cache_map_uncached(CUtensorMap* map, const void* base, int B, int Lmax, int Hkv, int D, int box_keys);
 static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, int Hkv, int D, int box_keys) {
+    const MapKey key{base, 1, B, Lmax, Hkv, D, box_keys};
+    if (cached_map(key, map, nullptr)) return SWAA_OK;
+    const int rc = make_cache_map_uncached(map, base, B, Lmax, Hkv, D, box_keys);
+    if (rc == SWAA_OK) cached_map(key, nullptr, map);
+    return rc;
+}
+static int make_cache_map_uncached(CUtensorMap* map, const void* base, int B, int Lmax, int Hkv, int D, int box_keys) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return SWAA_ERR_CUDA;
     const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)Lmax, (cuuint64_t)B};
@@ -135,12 +180,22 @@ static int make_cache_map(CUtensorMap* map, const void* base, int B, int Lmax, i
     return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
+// The dynamic shared-memory limit of a kernel instance is set once per device (it is a per-device function attribute).
+template <typename Kernel>
+static int ensure_dynamic_smem(Kernel kernel, int bytes, std::atomic<bool> (&done)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SWAA_ERR_CUDA;
+    if (done[dev].load(std::memory_order_acquire)) return SWAA_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return SWAA_ERR_CUDA;
+    done[dev].store(true, std::memory_order_release);
+    return SWAA_OK;
+}
+
 template <int D, int NH, bool kPaged, bool kShard = false>
 static int launch_decode(const CUtensorMap (&tm)[4], const DecodeParams& p, int blocks, cudaStream_t st) {
     using L = DecodeSmem<D, NH>;
-    if (cudaFuncSetAttribute(decode_kernel<D, NH, kPaged, kShard>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             L::kDynamicBytes) != cudaSuccess)
-        return SWAA_ERR_CUDA;
+    static std::atomic<bool> attr_done[64];
+    if (ensure_dynamic_smem(decode_kernel<D, NH, kPaged, kShard>, L::kDynamicBytes, attr_done) != SWAA_OK) return SWAA_ERR_CUDA;
     decode_kernel<D, NH, kPaged, kShard><<<(unsigned)blocks, kDecodeThreads, L::kDynamicBytes, st>>>(tm[0], tm[1], tm[2], tm[3], p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
@@ -327,7 +382,15 @@ namespace swaa {
 
 // Tensor map over a token-major bf16 tensor [T, H, D]: dimensions (D, H, T) innermost first; one box is
 // [128 tokens] x [1 head] x [64 channels] = 128 rows of 128 bytes, written with the 128-byte swizzle.
+static int make_token_major_map_uncached(CUtensorMap* map, const void* base, int T, int H, int D, int box_tokens);
 static int make_token_major_map(CUtensorMap* map, const void* base, int T, int H, int D, int box_tokens = 128) {
+    const MapKey key{base, 2, T, H, D, box_tokens, 0};
+    if (cached_map(key, map, nullptr)) return SWAA_OK;
+    const int rc = make_token_major_map_uncached(map, base, T, H, D, box_tokens);
+    if (rc == SWAA_OK) cached_map(key, nullptr, map);
+    return rc;
+}
+static int make_token_major_map_uncached(CUtensorMap* map, const void* base, int T, int H, int D, int box_tokens) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return SWAA_ERR_CUDA;
     const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T};
@@ -354,18 +417,17 @@ static int make_accum_map(CUtensorMap* map, const float* base, int T, int H, int
     return r == CUDA_SUCCESS ? SWAA_OK : SWAA_ERR_CUDA;
 }
 
-template <int D, int kMode>
+template <int D, int kMode, bool kLseOnly = false>
 static int launch_prefill(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                           const CUtensorMap& tsk, const CUtensorMap& tsv, const PrefillParams& p, int sm_count,
                           cudaStream_t st) {
     using L = PrefillSmem<D>;
-    if (cudaFuncSetAttribute(prefill_kernel<D, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             L::kDynamicBytes) != cudaSuccess)
-        return SWAA_ERR_CUDA;
+    static std::atomic<bool> attr_done[64];
+    if (ensure_dynamic_smem(prefill_kernel<D, kMode, kLseOnly>, L::kDynamicBytes, attr_done) != SWAA_OK) return SWAA_ERR_CUDA;
     // persistent blocks: one per SM (or fewer when there is less work), each walks its share of the items
     long long blocks = (long long)p.n_pairs * p.tiles_ub;
     if (blocks > sm_count) blocks = sm_count;
-    prefill_kernel<D, kMode><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, tsk, tsv, p);
+    prefill_kernel<D, kMode, kLseOnly><<<(unsigned)blocks, kPrefillThreads, L::kDynamicBytes, st>>>(tq, tk, tv, to, tsk, tsv, p);
     launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? SWAA_OK : SWAA_ERR_CUDA;
 }
@@ -385,6 +447,7 @@ struct PrefillExtras {
     const uint8_t* is_full_seq = nullptr;  // mask policy per sequence (chunked / paged)
     // context-parallel prefill: local keys start at key_pos0[b]; sink rows in [B, sink_rows, Hkv, D] buffers
     bool context_parallel = false;
+    bool lse_only = false;  // chunked layout only: write lse and nothing else (q, k needed; v and out are not touched)
     const int32_t* key_pos0 = nullptr;
     const void* sink_k = nullptr;
     const void* sink_v = nullptr;
@@ -400,6 +463,11 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
     if ((!is_full || ex.is_full_seq != nullptr) && window < 1) return SWAA_ERR_INVALID_ARG;
     if (Hq % Hkv != 0 || (D != 64 && D != 128)) return SWAA_ERR_UNSUPPORTED;
     if (B == 0 || Tq == 0) return SWAA_OK;
+    if (ex.lse_only) {  // v and out stand in with q's address: never dereferenced, only encoded into unused tensor maps
+        if (!lse || !cu_seqlens_k || paged.block_table || ex.context_parallel) return SWAA_ERR_INVALID_ARG;
+        v = k;
+        out = const_cast<void*>(q);
+    }
     if (!q || !k || !v || !out || !cu_seqlens_q) return SWAA_ERR_INVALID_ARG;
     if (ex.context_parallel) {
         if (!ex.key_pos0 || ex.sink_rows < 0 || (reinterpret_cast<uintptr_t>(ex.key_pos0) & 3u) != 0)
@@ -483,6 +551,9 @@ static int prefill_impl(const void* q, const void* k, const void* v, void* out, 
     if (is_paged)
         return D == 128 ? launch_prefill<128, 2>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st)
                         : launch_prefill<64, 2>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st);
+    if (ex.lse_only)
+        return D == 128 ? launch_prefill<128, 1, true>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st)
+                        : launch_prefill<64, 1, true>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st);
     if (cu_seqlens_k != nullptr)
         return D == 128 ? launch_prefill<128, 1>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st)
                         : launch_prefill<64, 1>(tq, tk, tv, to, tsk, tsv, p, info.sm_count, st);
@@ -740,15 +811,19 @@ extern "C" int swaa_lazy_ratio(const void* q, const void* k, const void* v, cons
                                const int32_t* cu_seqlens_k, int B, int Tq, int Tk, int max_seqlen_q, int max_seqlen_k,
                                int Hq, int Hkv, int D, int recent, int n_sink, float scale, float* ratio,
                                void* scratch_out, float* scratch_lse, void* stream) {
-    if (!ratio || !scratch_out || !scratch_lse || !cu_seqlens_k) return SWAA_ERR_INVALID_ARG;
+    (void)v;            // the probe needs no values: both passes run the kernel instance that only forms log-sum-exps
+    (void)scratch_out;
+    if (!ratio || !scratch_lse || !cu_seqlens_k) return SWAA_ERR_INVALID_ARG;
     if (recent < 1 || B < 1 || Tq < 1) return SWAA_ERR_INVALID_ARG;
     float* lse_recent = scratch_lse;
     float* lse_full = scratch_lse + (size_t)Hq * Tq;
-    int rc = prefill_impl(q, k, v, scratch_out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq,
-                          Hkv, D, recent, n_sink, 0, scale, lse_recent, stream);
+    PrefillExtras ex;
+    ex.lse_only = true;
+    int rc = prefill_impl(q, k, nullptr, nullptr, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq,
+                          Hkv, D, recent, n_sink, 0, scale, lse_recent, stream, PagedKV(), ex);
     if (rc != SWAA_OK) return rc;
-    rc = prefill_impl(q, k, v, scratch_out, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq, Hkv, D,
-                      1, 0, 1, scale, lse_full, stream);
+    rc = prefill_impl(q, k, nullptr, nullptr, cu_seqlens_q, cu_seqlens_k, B, Tq, Tk, max_seqlen_q, max_seqlen_k, Hq, Hkv, D,
+                      1, 0, 1, scale, lse_full, stream, PagedKV(), ex);
     if (rc != SWAA_OK) return rc;
     lazy_ratio_reduce_kernel<<<(unsigned)Hq, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(lse_recent, lse_full, Tq,
                                                                                                 ratio);

@@ -245,7 +245,10 @@ struct WorkItem {
 // 3: context-parallel prefill, mode 1 with the local keys starting at position key_pos0[b] of their sequence and the
 // sink keys before that position read from a separate buffer (tm_sk, tm_sv) as leading key tiles of the item.
 // The self-attention instance compiles the offsets away.
-template <int D, int kMode>
+// kLseOnly: only the log-sum-exp of every row is wanted (the lazy-ratio probe): no V tiles are fetched, no P V product
+// is issued, P is not formed and nothing is written to `out`; the barrier protocol stays the same, with "P ready"
+// meaning "S has been read" and the V-tile barriers completed by a plain arrival.
+template <int D, int kMode, bool kLseOnly = false>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -468,6 +471,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         mbar_wait(bar(BAR_KF + s), ph, abort_flag);  // the K copy just issued
                         break;
                     }
+                    if (kLseOnly) {
+                        mbar_arrive(bar(BAR_VF + s));  // no V tile: complete the stage's barrier by hand
+                        continue;
+                    }
                     mbar_arrive_expect_tx(bar(BAR_VF + s), (uint32_t)L::kTileBytes);
 #pragma unroll
                     for (int pn = 0; pn < L::kPanels; ++pn) {
@@ -598,7 +605,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (ok && n == 0) ok = mbar_wait(bar(BAR_OF + 0), ((uint32_t)items_side[0] & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(0, sv, n > 0);
+                    if (!kLseOnly) issue_pv(0, sv, n > 0);
                     // O-done is only waited for by the item's epilogue: between tiles the S-full barrier of tile n + 1
                     // already implies PV(n) (a commit covers every product issued before it), and every commit costs
                     // this thread some 40 cycles
@@ -614,7 +621,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                             ok = mbar_wait(bar(BAR_OF + 1), ((uint32_t)items_side[1] & 1u) ^ 1u, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_pv(1, sv, n > 0);
+                        if (!kLseOnly) issue_pv(1, sv, n > 0);
                         if (!has_next) tc_commit(bar(BAR_OD + 1));
                         ++gs[1];
                         if (has_next) {
@@ -690,6 +697,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 tmem_ld32(tS + 64, sr + 64);
                 tmem_ld32(tS + 96, sr + 96);
                 tc_wait_ld();
+                if (kLseOnly) {  // S is in registers: the next Q K^T of this side may overwrite it
+                    tc_fence_before();
+                    mbar_arrive(bar(BAR_PR + side));
+                }
                 uint32_t vis[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
                 if (need_mask) {
                     // Bit b of vis[cc] <=> column c = 32*cc + b of this tile is visible to this row:
@@ -725,7 +736,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     // previous tile has completed: it was issued before the QK whose S-full barrier this warp passed
                     const float alpha = (m_used == -INFINITY) ? 1.f : ex2f((m_used - m_new) * p.sl2);
 #pragma unroll
-                    for (int cc = 0; cc < D / 32; ++cc) {
+                    for (int cc = 0; cc < (kLseOnly ? 0 : D / 32); ++cc) {
                         uint32_t orr[32];
                         tmem_ld32(tO + cc * 32, orr);
                         tc_wait_ld();
@@ -733,7 +744,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
                         tmem_st32(tO + cc * 32, orr);
                     }
-                    tc_wait_st();
+                    if (!kLseOnly) tc_wait_st();
                     l_sum *= alpha;
                     m_used = m_new;
                 } else if (m_used == -INFINITY) {
@@ -749,7 +760,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         // no row of this warp sees any of these 32 keys: P = 0 without touching the MUFU
 #pragma unroll
                         for (int c = 0; c < 16; ++c) pk[c] = 0u;
-                        tmem_st16(tS + cc * 16, pk);
+                        if (!kLseOnly) tmem_st16(tS + cc * 16, pk);
                         continue;
                     }
 #pragma unroll
@@ -768,18 +779,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         }
                         if (c & 1) psum_b = add_f32x2(psum_b, pack_f32x2(p0, p1));
                         else psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
-                        pk[c] = pack_bf16x2(p0, p1);
+                        if (!kLseOnly) pk[c] = pack_bf16x2(p0, p1);
                     }
-                    tmem_st16(tS + cc * 16, pk);
+                    if (!kLseOnly) tmem_st16(tS + cc * 16, pk);
                 }
                 {
                     float a0, a1;
                     unpack_f32x2(add_f32x2(psum_a, psum_b), a0, a1);
                     l_sum += a0 + a1;
                 }
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(bar(BAR_PR + side));
+                if (!kLseOnly) {
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bar(BAR_PR + side));
+                }
             }
             if (!ok) break;
             // ---- epilogue of this item: O / l -> bf16 -> global
@@ -788,13 +801,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ++items_done;
             tc_fence_after();
             uint32_t orr[D];
+            if (!kLseOnly) {
 #pragma unroll
-            for (int cc = 0; cc < D / 32; ++cc) tmem_ld32(tO + cc * 32, orr + cc * 32);
-            tc_wait_ld();
+                for (int cc = 0; cc < D / 32; ++cc) tmem_ld32(tO + cc * 32, orr + cc * 32);
+                tc_wait_ld();
+            }
             tc_fence_before();
             mbar_arrive(bar(BAR_OF + side));  // O may be overwritten by the next item's first PV
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            if (q0 + wq * 32 + 31 < seq_len) {
+            if (kLseOnly) {
+                // nothing to store but the log-sum-exp below
+            } else if (q0 + wq * 32 + 31 < seq_len) {
                 // all 32 rows of this warp are valid: stage [32 rows][64 ch] panels in shared memory in the
                 // 128-byte-swizzled layout and let TMA write them (fully coalesced, off the LSU path)
                 const uint32_t stage = sStage + (uint32_t)warp * 4096u;

@@ -131,10 +131,15 @@ def test_lazy_ratio_matches_oracle():
         q, k, v = make(lq, lk, Hq, Hkv, D, seed=123)
         q = (q.float() * 2.0).to(torch.bfloat16)  # sharper softmax: the ratio is not just a key count
         ratio = torch.full((Hq,), float("nan"), device="cuda")
-        so = torch.empty_like(q)
         sl = torch.empty((2, Hq, sum(lq)), dtype=torch.float32, device="cuda")
-        swaa.swaa_lazy_ratio(q, k, v, _cu(lq), _cu(lk), max(lq), max(lk), recent, S, ratio, so, sl)
+        # the probe needs neither values nor an attention output: both may be left out
+        swaa.swaa_lazy_ratio(q, k, None, _cu(lq), _cu(lk), max(lq), max(lk), recent, S, ratio, None, sl)
         assert swaa.last_device_status() == 0
+        # its two log-sum-exp passes against the oracle's (windowed + sinks, then full causal)
+        for idx, (W_, S_, full_) in enumerate(((recent, S, False), (1, 0, True))):
+            want = oracle.prefill_chunked(inputs.to_f32_numpy(q), inputs.to_f32_numpy(k), inputs.to_f32_numpy(k),
+                                          _cu(lq).cpu().numpy(), _cu(lk).cpu().numpy(), W_, S_, full_)["lse"]
+            np.testing.assert_allclose(sl[idx].cpu().numpy().T, want, rtol=0, atol=2e-3)
         ref = oracle.lazy_ratio(inputs.to_f32_numpy(q), inputs.to_f32_numpy(k), None, _cu(lq).cpu().numpy(),
                                 _cu(lk).cpu().numpy(), recent, S)
         got = ratio.cpu().numpy()
