@@ -33,13 +33,14 @@ METRIC = "swa_prefill_effective_tflops"
 UNIT = "TFLOP/s"
 L2_FLUSH_BYTES = 256 << 20
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (None until a capture exists).
-PREFILL_DRAM_TRAFFIC_BYTES = 642869504  # 404.54 MB read + 238.33 MB written, profiles/prefill_kernel_cfg2_long_swa.txt
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (first of
+# the two captured launches each; taken on the kernels as committed).
+PREFILL_DRAM_TRAFFIC_BYTES = 403651840 + 234990848  # profiles/prefill_kernel_cfg2_long_swa.txt
 
-# decode kernel: 4 x (1.0739 GB read + 4 MB written) scaled from the B=4 capture; 270.0 MB + 5 MB at full size
-DECODE_FA_DRAM_TRAFFIC_BYTES = 4 * (1073919000 + 4249600)
-DECODE_SWA_DRAM_TRAFFIC_BYTES = 269955584 + 4963840
+# FA decode: 4 x the B=4 capture (traffic grows in proportion to B), profiles/decode_kernel_fa_quarter_of_cfg4.txt;
+# SWA decode: full size, profiles/decode_kernel_swa_cfg4.txt
+DECODE_FA_DRAM_TRAFFIC_BYTES = 4 * (1073921000 + 3599104)
+DECODE_SWA_DRAM_TRAFFIC_BYTES = 269949440 + 3997696
 
 
 def visible_pairs(L, W, S, full):
