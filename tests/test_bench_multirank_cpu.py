@@ -54,6 +54,21 @@ dist.destroy_process_group()
 """
 
 
+def _json_objects(text):
+    """Every JSON object printed on stdout; two ranks that print at the same moment can end up on one line."""
+    dec, out = json.JSONDecoder(), []
+    for line in text.splitlines():
+        i = line.find("{")
+        while i >= 0:
+            try:
+                obj, end = dec.raw_decode(line, i)
+            except json.JSONDecodeError:
+                break
+            out.append(obj)
+            i = line.find("{", end)
+    return out
+
+
 def _free_port():
     import socket
     with socket.socket() as sk:
@@ -73,7 +88,7 @@ def test_two_rank_timing_reduction(tmp_path):
     script.write_text(WORKER)
     r = _launch([str(script)])
     assert r.returncode == 0, r.stderr[-2000:]
-    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    lines = _json_objects(r.stdout)
     assert sorted(d["rank"] for d in lines) == [0, 1]
     for d in lines:
         assert d["red"] == [11.0, 5.0, 1.0]                # element-wise max over the two ranks, on every rank
@@ -84,7 +99,7 @@ def test_reference_arm_prints_from_rank_zero_only():
     r = _launch(["bench.py", "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0"],
                 env_extra={"OMP_NUM_THREADS": "2"}, timeout=600)
     assert r.returncode == 0, r.stderr[-2000:]
-    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    lines = _json_objects(r.stdout)
     assert len(lines) == 1
     d = lines[0]
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
@@ -99,7 +114,7 @@ def test_two_rank_gather_of_decode_partials(tmp_path):
     script.write_text(SPLIT_WORKER)
     r = _launch([str(script)], env_extra={"OMP_NUM_THREADS": "2"})
     assert r.returncode == 0, r.stderr[-2000:]
-    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    lines = _json_objects(r.stdout)
     assert sorted(d["rank"] for d in lines) == [0, 1]
     for d in lines:
         assert d["err"]["False"] < 1e-13 and d["err"]["True"] < 1e-13
