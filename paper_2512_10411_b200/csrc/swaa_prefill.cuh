@@ -139,10 +139,13 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 // x = n + f with n = round(x), f in [-1/2, 1/2]; 2^f by a cubic with constant term exactly 1 (minimax fit of
 // the other three coefficients: relative error 1.0e-4, far below the bf16 rounding of P), so that 2^0 = 1
 // exactly as on the special-function unit and a row of equal scores sums to its key count; n is added into
-// the exponent field.  Arguments below -126 (masked scores arrive as -inf) give exactly 0, as
-// ex2.approx.ftz does.
+// the exponent field.  The argument is first raised to -127, where the result is exactly 0 (f = 0, the cubic gives
+// 1.0 and the exponent field cancels), so masked scores (-inf) and anything below 2^-127 give exact zeros as
+// ex2.approx.ftz does, at the price of one max per element instead of a compare and a select.
 __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, float& r1) {
     const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    x0 = fmaxf(x0, -127.f);
+    x1 = fmaxf(x1, -127.f);
     const uint64_t xx = pack_f32x2(x0, x1);
     uint64_t t, fl, f, q;
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(t) : "l"(xx), "l"(pack_f32x2(kMagic, kMagic)));
@@ -155,12 +158,13 @@ __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& r0, floa
     float t0, t1, q0, q1;
     unpack_f32x2(t, t0, t1);
     unpack_f32x2(q, q0, q1);
-    r0 = x0 < -126.f ? 0.f : __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
-    r1 = x1 < -126.f ? 0.f : __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+    r0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    r1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
 }
 
-// Bit c (0..15) set: column pair c of every 32-column chunk of a score tile takes the polynomial path.
-constexpr uint32_t kPolyPairMask = 0x8080u;
+// Bit c (0..15) set: column pair c of every 32-column chunk of a score tile takes the polynomial path: a quarter
+// of the exponentials (measured best among 1/8, 3/16, 1/4, 5/16, 1/2, 3/4 and several placements).
+constexpr uint32_t kPolyPairMask = 0x8888u;
 
 #define SWAA_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
 #define SWAA_I8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
