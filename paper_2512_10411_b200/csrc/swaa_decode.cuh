@@ -656,14 +656,34 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                             num += wgt * os[i];
                         }
                     } else {
-                        for (int cc = c_first; cc <= c_last; ++cc)
-                            M = fmaxf(M, __ldcg(p.part + ((size_t)slot_of(cc) * HC + hh) * (D + 2)));
-                        for (int cc = c_first; cc <= c_last; ++cc) {
-                            const float* pp = p.part + ((size_t)slot_of(cc) * HC + hh) * (D + 2);
-                            const float ms = __ldcg(pp);
-                            const float wgt = ms == -INFINITY ? 0.f : ex2f((ms - M) * p.sl2);
-                            den += wgt * __ldcg(pp + 1);
-                            num += wgt * __ldcg(pp + 2 + d);
+                        // many parts (a long item of a small batch): eight partials per round trip to L2, merged
+                        // into a running (max, sum, O) -- loads one by one would cost a round trip each
+                        for (int c0 = c_first; c0 <= c_last; c0 += 8) {
+                            float ms[8], ls[8], os[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                ms[i] = -INFINITY;
+                                ls[i] = os[i] = 0.f;
+                                if (c0 + i <= c_last) {
+                                    const float* pp = p.part + ((size_t)slot_of(c0 + i) * HC + hh) * (D + 2);
+                                    ms[i] = __ldcg(pp);
+                                    ls[i] = __ldcg(pp + 1);
+                                    os[i] = __ldcg(pp + 2 + d);
+                                }
+                            }
+                            float Mn = M;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) Mn = fmaxf(Mn, ms[i]);
+                            const float keep = M == -INFINITY ? 0.f : ex2f((M - Mn) * p.sl2);
+                            den *= keep;
+                            num *= keep;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const float wgt = ms[i] == -INFINITY ? 0.f : ex2f((ms[i] - Mn) * p.sl2);
+                                den += wgt * ls[i];
+                                num += wgt * os[i];
+                            }
+                            M = Mn;
                         }
                     }
                     if (kShard) {
