@@ -35,12 +35,12 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (first of
 # the two captured launches each; taken on the kernels as committed).
-PREFILL_DRAM_TRAFFIC_BYTES = 403651840 + 234990848  # profiles/prefill_kernel_cfg2_long_swa.txt
+PREFILL_DRAM_TRAFFIC_BYTES = 404261888 + 235476224  # profiles/prefill_kernel_cfg2_long_swa.txt
 
 # FA decode: 4 x the B=4 capture (traffic grows in proportion to B), profiles/decode_kernel_fa_quarter_of_cfg4.txt;
 # SWA decode: full size, profiles/decode_kernel_swa_cfg4.txt
-DECODE_FA_DRAM_TRAFFIC_BYTES = 4 * (1073921000 + 3599104)
-DECODE_SWA_DRAM_TRAFFIC_BYTES = 269949440 + 3997696
+DECODE_FA_DRAM_TRAFFIC_BYTES = 4 * (1073863000 + 3872512)
+DECODE_SWA_DRAM_TRAFFIC_BYTES = 269665536 + 4531200
 
 
 def visible_pairs(L, W, S, full):
