@@ -234,6 +234,117 @@ def gather_decode_partials(part, world):
     return out
 
 
+def exchange_halo_and_sinks(k_own, v_own, window, n_sink, rank, world):
+    """The data movement of a context-parallel SWA prefill for one sequence cut into `world` equal stretches: rank r
+    owns k_own, v_own [L / world, Hkv, D] (positions r * L / world ...).  It receives the last window - 1 rows of rank
+    r - 1 (one neighbour send; the stretch must be at least that long) and the first n_sink rows of rank 0 (one
+    broadcast).  Returns (k_local, v_local, sink_k, sink_v, key_pos0): halo ++ own stretch, the sink rows as
+    [1, max(n_sink, 1), Hkv, D], and the position of the first local key -- the arguments of
+    swaa_prefill_context_parallel."""
+    import torch
+    import torch.distributed as dist
+
+    own = k_own.shape[0]
+    halo = min(window - 1, own) if rank > 0 else 0
+    if world > 1 and window - 1 > own:
+        raise ValueError("the stretch of a rank must hold at least window - 1 tokens")
+    sink_rows = max(n_sink, 1)
+    sink_k = torch.zeros((1, sink_rows) + tuple(k_own.shape[1:]), dtype=k_own.dtype, device=k_own.device)
+    sink_v = torch.zeros_like(sink_k)
+    if rank == 0:
+        m = min(sink_rows, own)
+        sink_k[0, :m] = k_own[:m]
+        sink_v[0, :m] = v_own[:m]
+    if world == 1:
+        return k_own, v_own, sink_k, sink_v, 0
+    dist.broadcast(sink_k, src=0)
+    dist.broadcast(sink_v, src=0)
+    send_rows = min(window - 1, own)
+    k_local = torch.empty((halo + own,) + tuple(k_own.shape[1:]), dtype=k_own.dtype, device=k_own.device)
+    v_local = torch.empty_like(k_local)
+    k_local[halo:] = k_own
+    v_local[halo:] = v_own
+    ops = []
+    if rank + 1 < world:
+        ops += [dist.P2POp(dist.isend, k_own[own - send_rows:].contiguous(), rank + 1),
+                dist.P2POp(dist.isend, v_own[own - send_rows:].contiguous(), rank + 1)]
+    if rank > 0:
+        hk = torch.empty((halo,) + tuple(k_own.shape[1:]), dtype=k_own.dtype, device=k_own.device)
+        hv = torch.empty_like(hk)
+        ops += [dist.P2POp(dist.irecv, hk, rank - 1), dist.P2POp(dist.irecv, hv, rank - 1)]
+    if ops:
+        for req in dist.batch_isend_irecv(ops):
+            req.wait()
+    if rank > 0:
+        k_local[:halo] = hk
+        v_local[:halo] = hv
+    return k_local, v_local, sink_k, sink_v, rank * own - halo
+
+
+def run_context_parallel(args, rank, local_rank, world):
+    """Workload 2 (SWA prefill, L=32768) cut along the context over the ranks (strong scaling): halo and sink rows are
+    moved by exchange_halo_and_sinks, then every rank runs swaa_prefill_context_parallel on its stretch.  The two parts
+    are timed separately; with one rank there is nothing to move."""
+    import torch
+
+    import paper_2512_10411_b200 as swaa
+    from paper_2512_10411_b200 import inputs
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    cfg = inputs.cfg_long()
+    L = cfg.seqlens[0]
+    q, k, v, _ = inputs.make_prefill_inputs(cfg, dev)   # every rank draws the same sequence and keeps its stretch
+    own = L // world
+    sl = slice(rank * own, (rank + 1) * own)
+    q_own, k_own, v_own = q[sl].contiguous(), k[sl].contiguous(), v[sl].contiguous()
+    del q, k, v
+    out = torch.empty_like(q_own)
+    cu_q = torch.tensor([0, own], dtype=torch.int32, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_rd = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    t_x, t_k = [], []
+    for it in range(max(args.warmup, 3) + args.steps):
+        flush.zero_()
+        flush_rd.sum()
+        if world > 1:
+            dist.barrier()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(stream)
+        k_loc, v_loc, sk, sv, p0 = exchange_halo_and_sinks(k_own, v_own, cfg.window, cfg.n_sink, rank, world)
+        e[1].record(stream)
+        cu_k = torch.tensor([0, k_loc.shape[0]], dtype=torch.int32, device=dev)
+        pos0 = torch.tensor([p0], dtype=torch.int32, device=dev)
+        swaa.swaa_prefill_context_parallel(q_own, k_loc, v_loc, sk, sv, out, cu_q, cu_k, pos0, own, k_loc.shape[0],
+                                           cfg.window, cfg.n_sink)
+        e[2].record(stream)
+        torch.cuda.synchronize()
+        if it >= max(args.warmup, 3):
+            t_x.append(e[0].elapsed_time(e[1]))
+            t_k.append(e[1].elapsed_time(e[2]))
+    assert swaa.last_device_status() == 0
+    med_x, med_k = max_over_ranks([stats_ms(t_x)["median"], stats_ms(t_k)["median"]], world, dev)
+    flops = 4.0 * cfg.D * cfg.Hq * visible_pairs(L, cfg.window, cfg.n_sink, False)
+    if rank == 0:
+        tf = flops / ((med_x + med_k) * 1e-3) / 1e12
+        print(json.dumps({"metric": METRIC, "value": tf, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                          "warmup": max(args.warmup, 3), "ms_per_step": med_x + med_k, "higher_is_better": True,
+                          "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                          "config": {"workload": f"cfg2 long-context SWA prefill cut along the context over {world} rank(s)",
+                                     "l2": "flushed before every step"},
+                          "context_parallel": {"exchange_ms": med_x, "kernel_ms": med_k,
+                                               "kernel_tflops_all_ranks": flops / (med_k * 1e-3) / 1e12,
+                                               "frac_of_measured_peak_per_gpu": flops / world / (med_k * 1e-3) / 1e12 / peaks["bf16_tflops"]}}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_decode_split(args, rank, local_rank, world):
     """Decode workload 4 with the cache cut along the context over the ranks (strong scaling: the job is one decode
     step of the whole batch).  Rank r holds positions [r * Lmax / N, (r + 1) * Lmax / N) of every sequence; a step is
@@ -821,6 +932,9 @@ def main():
                     help="decode workload 4 with the cache cut along the context over the ranks (or, on one GPU, over "
                          "--shards shards run in sequence) and exit")
     ap.add_argument("--shards", type=int, default=4)
+    ap.add_argument("--context-parallel", action="store_true",
+                    help="SWA prefill of workload 2 cut along the context over the ranks (halo + sink exchange, then "
+                         "swaa_prefill_context_parallel) and exit")
     ap.add_argument("--sweep", action="store_true",
                     help="time swaa_prefill on the other workloads and the L / W / n_sink sweeps (one GPU) and exit")
     args = ap.parse_args()
@@ -833,7 +947,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.decode_split:
+    if args.context_parallel:
+        run_context_parallel(args, rank, local_rank, world)
+    elif args.decode_split:
         run_decode_split(args, rank, local_rank, world)
     elif args.impl == "reference":
         run_reference(args, rank)

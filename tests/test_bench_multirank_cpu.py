@@ -54,6 +54,38 @@ dist.destroy_process_group()
 """
 
 
+HALO_WORKER = r"""
+import os, sys, json
+sys.path.insert(0, os.environ["SWAA_ROOT"])
+import numpy as np, torch
+import torch.distributed as dist
+import bench, oracle
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+L, Hq, Hkv, D = 96, 4, 2, 8
+g = torch.Generator().manual_seed(9)                       # every rank draws the same sequence and keeps its stretch
+q = torch.randn((L, Hq, D), generator=g).to(torch.bfloat16).float()
+k = torch.randn((L, Hkv, D), generator=g).to(torch.bfloat16).float()
+v = torch.randn((L, Hkv, D), generator=g).to(torch.bfloat16).float()
+own = L // world
+sl = slice(rank * own, (rank + 1) * own)
+res = {}
+for W, S in ((17, 3), (48, 0), (5, 9)):
+    kl, vl, sk, sv, p0 = bench.exchange_halo_and_sinks(k[sl].contiguous(), v[sl].contiguous(), W, S, rank, world)
+    assert p0 == max(0, rank * own - (W - 1)) and kl.shape[0] == (rank + 1) * own - p0
+    got = oracle.prefill_cp(q[sl].numpy(), kl.numpy(), vl.numpy(), sk.numpy(), sv.numpy(), [0, own], [0, kl.shape[0]], [p0], W, S, False)
+    want = oracle.prefill(q.numpy(), k.numpy(), v.numpy(), [0, L], W, S, False)
+    res[f"{W},{S}"] = bool(np.array_equal(got["out"], want["out"][sl]) and np.array_equal(got["nvis"], want["nvis"][sl]))
+try:
+    bench.exchange_halo_and_sinks(k[sl].contiguous(), v[sl].contiguous(), own + 2, 0, rank, world)
+    res["short"] = False
+except ValueError:
+    res["short"] = True
+print(json.dumps({"rank": rank, "ok": res}), flush=True)
+dist.destroy_process_group()
+"""
+
+
 def _json_objects(text):
     """Every JSON object printed on stdout; two ranks that print at the same moment can end up on one line."""
     dec, out = json.JSONDecoder(), []
@@ -118,3 +150,17 @@ def test_two_rank_gather_of_decode_partials(tmp_path):
     assert sorted(d["rank"] for d in lines) == [0, 1]
     for d in lines:
         assert d["err"]["False"] < 1e-13 and d["err"]["True"] < 1e-13
+
+
+def test_two_rank_halo_and_sink_exchange(tmp_path):
+    """The data movement of the context-parallel prefill over two gloo ranks: after the neighbour send of the halo and
+    the broadcast of the sink rows, every rank's stretch (computed with the oracle, on CPU) equals its rows of the
+    one-shot prefill bit for bit; a stretch shorter than the halo is refused."""
+    script = tmp_path / "halo_worker.py"
+    script.write_text(HALO_WORKER)
+    r = _launch([str(script)], env_extra={"OMP_NUM_THREADS": "2"})
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = _json_objects(r.stdout)
+    assert sorted(d["rank"] for d in lines) == [0, 1]
+    for d in lines:
+        assert all(d["ok"].values()), d
