@@ -667,11 +667,20 @@ def run_extra_workloads(swaa, torch, inputs, flush_l2, stream, peaks):
     1 (tiny), workload 5 (varlen), the time against L at fixed W (App. A: O(N * W)), and workload 3, the 36-layer
     interleaved stack with its mask policy from the layer schedule (per kind and in total; the stack runs for
     seconds, so its total is set against the sustained bf16 peak)."""
-    extra = {"note": "outside the timed step; median of `launches` launches each, L2 flushed before every launch"}
-    extra["cfg1_tiny"] = time_prefill_case(swaa, torch, flush_l2, stream, peaks, inputs.cfg_tiny(), False, 5)
-    extra["cfg5_varlen"] = time_prefill_case(swaa, torch, flush_l2, stream, peaks, inputs.cfg_varlen(), False, 3)
-    extra["linear_in_L"] = [time_prefill_case(swaa, torch, flush_l2, stream, peaks, inputs.cfg_long(L=L), False, 5)
-                            for L in (8192, 16384, 32768, 65536, 131072)]
+    extra = {"note": "outside the timed step; median of `launches` launches each, L2 flushed before every launch; the GPU "
+                     "idles for half a second before each case so that the power state of the case before it (the "
+                     "backward pass, the varlen batch) does not carry over; light cases first"}
+
+    def settled(*a, **kw):
+        torch.cuda.synchronize()
+        time.sleep(0.5)
+        return time_prefill_case(swaa, torch, flush_l2, stream, peaks, *a, **kw)
+
+    extra["cfg1_tiny"] = settled(inputs.cfg_tiny(), False, 5)
+    extra["linear_in_L"] = [settled(inputs.cfg_long(L=L), False, 5) for L in (8192, 16384, 32768, 65536, 131072)]
+    extra["cfg5_varlen"] = settled(inputs.cfg_varlen(), False, 3)
+    torch.cuda.synchronize()
+    time.sleep(0.5)
     pol = swaa.SwaaPolicy(n_layers=36, window=4096, n_sink=64, fa_start=3, fa_step=4, fa_decode=True)
     per_kind, flops = {False: [], True: []}, 0.0
     tensors = None
