@@ -8,7 +8,8 @@
 // that head's group); all query heads of a chunk are processed together so each K/V byte is fetched
 // once.  The visible cache entries of an item are cut into tiles of 64 keys (sink tiles, then window
 // tiles starting at the first window key).  All tiles of all items form one list in (sequence, item,
-// tile) order, and block c of a persistent grid (one block per SM) owns the contiguous run
+// tile) order, and block c of a persistent grid (at most one block per SM; the host prefers a block count that puts
+// the cuts on item boundaries, see plan_decode) owns the contiguous run
 // [c * tpc, (c+1) * tpc) of it, so every SM streams the same number of bytes whatever the batch
 // shape.  A block therefore holds at most two incomplete items (the first and the last of its run);
 // it writes complete items straight to `out` and incomplete ones as (max, sum, unnormalised O)
