@@ -227,7 +227,7 @@ struct PrefillSmem {
     static constexpr int kOffBar = kOffStage + 8 * 4096;
     // barriers: Q full/empty, K full/empty, V full/empty per stage, per side S-full / P-ready / O-done /
     // O-free, work-descriptor full/empty per slot, final, V-tile-cleared per stage (paged keys only)
-    static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1 + kStages;
+    static constexpr int kNumBars = 2 + 4 * kStages + 8 + 4 + 1 + kStages + 2;
     static constexpr int kOffMisc = kOffBar + kNumBars * 8;      // tmem slot, abort flag, work descriptors
     static constexpr int kBytes = kOffMisc + 128;
     static constexpr int kDynamicBytes = kBytes + 1024;          // room to align the base to 1024 B
@@ -281,7 +281,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // clear a stage twice before the issuer has waited for the first clear: reusing the stage needs the
     // issuer's V-empty commit, which follows that wait.
     constexpr int BAR_VC = BAR_FIN + 1;
-    static_assert(BAR_VC + ST == L::kNumBars, "barrier count");
+    // per side: the last quarter of P (keys 96..127) has been written; BAR_PR then stands for the first three quarters
+    constexpr int BAR_PQ = BAR_VC + ST;
+    static_assert(BAR_PQ + 2 == L::kNumBars, "barrier count");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + L::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* work_ring = reinterpret_cast<volatile int*>(tmem_slot + 4);  // 2 slots x 12 ints
@@ -294,6 +296,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int i = 0; i < L::kNumBars; ++i) {
             uint32_t count = 1u;
             if (i == BAR_PR || i == BAR_PR + 1 || i == BAR_OF || i == BAR_OF + 1) count = 128u;  // softmax threads
+            if (i == BAR_PQ || i == BAR_PQ + 1) count = 128u;
             if (i == BAR_WE || i == BAR_WE + 1) count = 10u;  // producer, issuer, one lane per softmax warp
             mbar_init(bar(i), count);
         }
@@ -551,10 +554,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     mma_ss_lh(d, qa + off, kb + off, desc_hi, kIdescQK, kk > 0 ? 1u : 0u);
                 }
             };
-            auto issue_pv = [&](int side, int stage, bool acc) {
+            auto issue_pv = [&](int side, int stage, bool acc, int kk0, int kk1) {
                 const uint32_t vb = pick(v_lo, stage), d = tO[side], a = tS[side];
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk) {
+                for (int kk = kk0; kk < kk1; ++kk) {
                     // P: 16 keys = 8 TMEM columns of packed bf16 pairs.  V: 16 key rows of 128 bytes.
                     mma_ts_lh(d, a + (uint32_t)kk * 8u, vb + (((uint32_t)kk * 2048u) >> 4), desc_hi, kIdescPV,
                               (acc || kk > 0) ? 1u : 0u);
@@ -609,7 +612,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     if (ok && n == 0) ok = mbar_wait(bar(BAR_OF + 0), ((uint32_t)items_side[0] & 1u) ^ 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    if (!kLseOnly) issue_pv(0, sv, n > 0);
+                    // the first three quarters of P are there: their products run while the softmax warps finish
+                    // the last quarter
+                    if (!kLseOnly) issue_pv(0, sv, n > 0, 0, 6);
+                    ok = mbar_wait(bar(BAR_PQ + 0), (uint32_t)gs[0] & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (!kLseOnly) issue_pv(0, sv, n > 0, 6, 8);
                     // O-done is only waited for by the item's epilogue: between tiles the S-full barrier of tile n + 1
                     // already implies PV(n) (a commit covers every product issued before it), and every commit costs
                     // this thread some 40 cycles
@@ -625,7 +634,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                             ok = mbar_wait(bar(BAR_OF + 1), ((uint32_t)items_side[1] & 1u) ^ 1u, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        if (!kLseOnly) issue_pv(1, sv, n > 0);
+                        if (!kLseOnly) issue_pv(1, sv, n > 0, 0, 6);
+                        ok = mbar_wait(bar(BAR_PQ + 1), (uint32_t)gs[1] & 1u, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (!kLseOnly) issue_pv(1, sv, n > 0, 6, 8);
                         if (!has_next) tc_commit(bar(BAR_OD + 1));
                         ++gs[1];
                         if (has_next) {
@@ -704,6 +717,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (kLseOnly) {  // S is in registers: the next Q K^T of this side may overwrite it
                     tc_fence_before();
                     mbar_arrive(bar(BAR_PR + side));
+                    mbar_arrive(bar(BAR_PQ + side));
                 }
                 uint32_t vis[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
                 if (need_mask) {
@@ -764,7 +778,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         // no row of this warp sees any of these 32 keys: P = 0 without touching the MUFU
 #pragma unroll
                         for (int c = 0; c < 16; ++c) pk[c] = 0u;
-                        if (!kLseOnly) tmem_st16(tS + cc * 16, pk);
+                        if (!kLseOnly) {
+                            tmem_st16(tS + cc * 16, pk);
+                            if (cc == 2) {  // three quarters of P written: hand them to the issuer
+                                tc_wait_st();
+                                tc_fence_before();
+                                mbar_arrive(bar(BAR_PR + side));
+                            }
+                        }
                         continue;
                     }
 #pragma unroll
@@ -785,7 +806,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                         else psum_a = add_f32x2(psum_a, pack_f32x2(p0, p1));
                         if (!kLseOnly) pk[c] = pack_bf16x2(p0, p1);
                     }
-                    if (!kLseOnly) tmem_st16(tS + cc * 16, pk);
+                    if (!kLseOnly) {
+                        tmem_st16(tS + cc * 16, pk);
+                        if (cc == 2) {  // three quarters of P written: hand them to the issuer
+                            tc_wait_st();
+                            tc_fence_before();
+                            mbar_arrive(bar(BAR_PR + side));
+                        }
+                    }
                 }
                 {
                     float a0, a1;
@@ -795,7 +823,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (!kLseOnly) {
                     tc_wait_st();
                     tc_fence_before();
-                    mbar_arrive(bar(BAR_PR + side));
+                    mbar_arrive(bar(BAR_PQ + side));
                 }
             }
             if (!ok) break;
