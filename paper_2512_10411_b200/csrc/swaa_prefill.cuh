@@ -18,7 +18,8 @@
 // P overwrite the first 64 columns of their own S and are consumed from TMEM as the A operand of
 // O += P V.  V tiles are used as the MN-major B operand exactly as TMA lands them.
 // Per key tile n the issuer runs  PV_A(n) QK_A(n+1) PV_B(n) QK_B(n+1), so the softmax of one side
-// overlaps the MMAs of the other.  The running maximum is only raised (and O rescaled) when it grows
+// overlaps the MMAs of the other; P arrives in two parts (keys 0..95, then 96..127) and the first six of the
+// eight P V instructions are issued on the first.  The running maximum is only raised (and O rescaled) when it grows
 // by more than 2^8; the final division by the row sum makes the result independent of that choice.
 //
 // Every wait is bounded: a wait that runs out records SWAA_ERR_TIMEOUT, all roles leave their loops,
