@@ -35,7 +35,7 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/ (first of
 # the two captured launches each; taken on the kernels as committed).
-PREFILL_DRAM_TRAFFIC_BYTES = 404261888 + 235476224  # profiles/prefill_kernel_cfg2_long_swa.txt
+PREFILL_DRAM_TRAFFIC_BYTES = 404582656 + 236282112  # profiles/prefill_kernel_cfg2_long_swa.txt
 
 # FA decode: 4 x the B=4 capture (traffic grows in proportion to B), profiles/decode_kernel_fa_quarter_of_cfg4.txt;
 # SWA decode: full size, profiles/decode_kernel_swa_cfg4.txt
