@@ -550,12 +550,54 @@ def run_ours(args, rank, local_rank, world):
         return a.elapsed_time(b) / n
 
     e2e_ms = time_loop(e2e_step, e2e_steps)
+
+    # The same steps pipelined over three streams with two sets of device buffers: the upload of step i + 1 and the
+    # download of step i - 1 run beside the kernel of step i (PCIe carries both directions at once).  Every step
+    # still uploads its own inputs and downloads its own result; only the waiting is overlapped.
+    def e2e_pipelined(n):
+        s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        bufs = [(q2, k2, v2, out), (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v), torch.empty_like(out))]
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_k = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        s_in.wait_event(a)
+        s_out.wait_event(a)
+        for i in range(n):
+            qd, kd, vd, od = bufs[i % 2]
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_k[i % 2])      # the kernel of step i - 2 has read these inputs
+                qd.copy_(qh, non_blocking=True)
+                kd.copy_(kh, non_blocking=True)
+                vd.copy_(vh, non_blocking=True)
+                ev_in[i % 2].record(s_in)
+            stream.wait_event(ev_in[i % 2])
+            if i >= 2:
+                stream.wait_event(ev_out[i % 2])      # the download of step i - 2 has read this output
+            swaa.swaa_prefill(qd, kd, vd, od, cu, L, pcfg.window, pcfg.n_sink, False)
+            ev_k[i % 2].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_k[i % 2])
+                outh.copy_(od, non_blocking=True)
+                ev_out[i % 2].record(s_out)
+        stream.wait_event(ev_out[(n - 1) % 2])
+        if n >= 2:
+            stream.wait_event(ev_out[(n - 2) % 2])
+        b.record(stream)
+        barrier()
+        del bufs
+        return a.elapsed_time(b) / n
+
+    e2e_pipe_ms = e2e_pipelined(max(6, e2e_steps))
     e2e_fa_ms = time_loop(lambda: e2e_decode_step(True, ws_fa), e2e_steps)
     e2e_swa_ms = time_loop(lambda: e2e_decode_step(False, ws_swa), e2e_steps)
 
     # ---------------------------------------------------------------- max over ranks
-    total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms = max_over_ranks(
-        [total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms], world, dev)
+    total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms, e2e_pipe_ms = max_over_ranks(
+        [total_ms, t_pre, t_fa, t_swa, e2e_ms, e2e_fa_ms, e2e_swa_ms, e2e_pipe_ms], world, dev)
     K, N = args.steps, world
 
 
@@ -629,9 +671,13 @@ def run_ours(args, rank, local_rank, world):
                    "value_from": "median over the timed steps of the prefill kernel time inside the step "
                                  "(CUDA events on the launching stream)"},
         "clocks": clocks,
-        "e2e": {"value": N * prefill_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+        "e2e": {"value": N * prefill_flops / (e2e_pipe_ms * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": int(q.numel() + k.numel() + v.numel()) * 2, "d2h_bytes_per_step": int(out.numel()) * 2,
-                "ms_per_step": e2e_ms},
+                "ms_per_step": e2e_pipe_ms,
+                "how": "every step uploads its Q, K, V from pinned host memory, runs swaa_prefill and downloads `out`; "
+                       "upload, kernel and download of neighbouring steps overlap (three streams, two device buffer sets)",
+                "serial": {"value": N * prefill_flops / (e2e_ms * 1e-3) / 1e12, "ms_per_step": e2e_ms,
+                           "how": "the same on one stream, nothing overlapped"}},
         "gpu_launches": int(launches),
         "roofline": {"kernel": "prefill_kernel<128, 0>", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
